@@ -1,0 +1,130 @@
+"""CPU oracle (fp64, plain definition) for the fused GEMM + epilogue + row-reduce operator.
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, the smoke check and the
+benchmark's CPU-baseline leg.  The CUDA package never imports it and shares no
+code with it.  The arithmetic lives in ``fgr_oracle.c`` (three nested loops);
+this file only compiles it with gcc and marshals numpy arrays through ctypes.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "fgr_oracle.c")
+_LIB = os.path.join(_HERE, "libfgr_oracle.so")
+
+F32, BF16 = 0, 1
+ACT_NONE, ACT_RELU, ACT_GELU_TANH = 0, 1, 2
+SCALE_NONE, SCALE_SCALAR, SCALE_PER_COLUMN = 0, 1, 2
+RED_LSE, RED_SOFTMAX, RED_MAXSUM, RED_MAX_SUMEXP = 0, 1, 2, 3
+
+
+class _Problem(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("M", ctypes.c_int32), ("N", ctypes.c_int32), ("K", ctypes.c_int32),
+                ("dtype", ctypes.c_int32), ("act", ctypes.c_int32), ("scale_kind", ctypes.c_int32),
+                ("reduce", ctypes.c_int32), ("scale", ctypes.c_double), ("bias_per_batch", ctypes.c_int32),
+                ("reserved", ctypes.c_int32)]
+
+
+def build(force: bool = False) -> str:
+    """Compiles ``fgr_oracle.c`` into ``libfgr_oracle.so`` next to it (gcc, strict fp64: no contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp%d" % os.getpid()
+        subprocess.run(["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fopenmp", "-fPIC", "-shared",
+                        "-o", tmp, _SRC, "-lm"], check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.fgr_oracle_rows.restype = ctypes.c_int
+        _lib.fgr_oracle_rows.argtypes = [ctypes.POINTER(_Problem)] + [ctypes.c_void_p] * 5 + [
+            ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int]
+        _lib.fgr_oracle_gelu_tanh.restype = ctypes.c_double
+        _lib.fgr_oracle_gelu_tanh.argtypes = [ctypes.c_double]
+        _lib.fgr_oracle_act.restype = ctypes.c_double
+        _lib.fgr_oracle_act.argtypes = [ctypes.c_int, ctypes.c_double]
+    return _lib
+
+
+def gelu_tanh(u: float) -> float:
+    return lib().fgr_oracle_gelu_tanh(float(u))
+
+
+def act(kind: int, u: float) -> float:
+    return lib().fgr_oracle_act(int(kind), float(u))
+
+
+def out_width(reduce: int) -> int:
+    return {RED_LSE: 1, RED_SOFTMAX: 0, RED_MAXSUM: 2, RED_MAX_SUMEXP: 2}[reduce]
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def run(X, W, bias, scale_vec, *, dtype, act, scale_kind, reduce, scale=1.0, bias_per_batch=0,
+        rows=None, want_y=True, nthreads=0):
+    """Evaluates the operator's definition in fp64.
+
+    X [batch, M, K] and W [batch, N, K] (2-D arrays are taken as batch 1): fp32 values
+    (``dtype == F32``) or uint16 bf16 bit patterns (``dtype == BF16``).  ``bias`` fp32 [N]
+    (or [batch, N] with ``bias_per_batch``) or None; ``scale_vec`` fp32 [N] or None.
+    ``rows``: global row indices (bt * M + m) to evaluate; None = all rows.
+
+    Returns ``(Y, out, threads)``: Y fp64 [nrows, N] (y, or P for SOFTMAX; None unless
+    ``want_y``), out fp64 [nrows, width] (None for SOFTMAX), threads used.
+    """
+    want = np.float32 if dtype == F32 else np.uint16
+    X = np.ascontiguousarray(X)
+    W = np.ascontiguousarray(W)
+    if X.dtype != want or W.dtype != want:
+        raise TypeError("X/W must be %s for dtype %d" % (want.__name__, dtype))
+    if X.ndim == 2:
+        X = X[None]
+    if W.ndim == 2:
+        W = W[None]
+    batch, M, K = X.shape
+    if W.shape[0] != batch or W.shape[2] != K:
+        raise ValueError("shape mismatch between X %s and W %s" % (X.shape, W.shape))
+    N = W.shape[1]
+    if bias is not None:
+        bias = np.ascontiguousarray(bias, dtype=np.float32).reshape(-1)
+        if bias.size != (batch * N if bias_per_batch else N):
+            raise ValueError("bias has %d elements" % bias.size)
+    if scale_vec is not None:
+        scale_vec = np.ascontiguousarray(scale_vec, dtype=np.float32).reshape(-1)
+        if scale_vec.size != N:
+            raise ValueError("scale_vec has %d elements" % scale_vec.size)
+    if rows is None:
+        nrows, rows_arr = batch * M, None
+    else:
+        rows_arr = np.ascontiguousarray(rows, dtype=np.int64).reshape(-1)
+        nrows = rows_arr.size
+    w = out_width(reduce)
+    need_y = want_y or reduce == RED_SOFTMAX
+    Y = np.empty((nrows, N), dtype=np.float64) if need_y else None
+    out = np.empty((nrows, w), dtype=np.float64) if w else None
+    prob = _Problem(batch, M, N, K, dtype, act, scale_kind, reduce, float(scale), int(bias_per_batch), 0)
+    rc = lib().fgr_oracle_rows(ctypes.byref(prob), _ptr(X), _ptr(W), _ptr(bias), _ptr(scale_vec), _ptr(rows_arr),
+                               nrows, _ptr(Y), _ptr(out), int(nthreads))
+    if rc < 0:
+        raise ValueError("fgr_oracle_rows rejected its arguments (code %d)" % rc)
+    return Y, out, rc
+
+
+def run_problem(p, rows=None, want_y=True, nthreads=0):
+    """``run`` on an object carrying X, W, bias, scale_vec and the descriptor fields as attributes."""
+    return run(p.X, p.W, p.bias, p.scale_vec, dtype=p.dtype, act=p.act, scale_kind=p.scale_kind,
+               reduce=p.reduce, scale=p.scale, bias_per_batch=p.bias_per_batch, rows=rows, want_y=want_y,
+               nthreads=nthreads)

@@ -1,0 +1,303 @@
+"""Pins for the CPU oracle: closed forms, invariants, brute force, hand-computed values and
+library routines.  None of these re-uses the oracle's own loop, so a dropped term, a wrong
+sign or index, or a transposed operand in the oracle fails at least one of them."""
+from decimal import Decimal, getcontext
+from fractions import Fraction
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import fgr_inputs as gi
+import oracle
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rand(shape, seed, tid=7, std=1.0):
+    return gi.normal(seed, tid, int(np.prod(shape)), std).reshape(shape)
+
+
+def _run(X, W, b, s, **kw):
+    kw.setdefault("dtype", oracle.F32)
+    kw.setdefault("act", oracle.ACT_NONE)
+    kw.setdefault("scale_kind", oracle.SCALE_NONE)
+    kw.setdefault("reduce", oracle.RED_LSE)
+    return oracle.run(X, W, b, s, **kw)
+
+
+# ---------------------------------------------------------------- hand-computed fixture
+def _golden(name):
+    for line in open(os.path.join(GOLDEN, "hand_2x2.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        k, *v = line.split()
+        if k == name:
+            return np.array([float(x) for x in v])
+    raise KeyError(name)
+
+
+@pytest.mark.parametrize("reduce,key", [(oracle.RED_MAXSUM, "maxsum"), (oracle.RED_LSE, "lse"),
+                                        (oracle.RED_MAX_SUMEXP, "max_sumexp"), (oracle.RED_SOFTMAX, "softmax")])
+def test_hand_example(reduce, key):
+    X = np.array([[1, 0], [1, 1]], dtype=np.float32)
+    W = np.array([[1, 2], [3, 4]], dtype=np.float32)
+    b = np.array([0, -1], dtype=np.float32)
+    s = np.array([2, 0.5], dtype=np.float32)
+    Y, out, _ = _run(X, W, b, s, act=oracle.ACT_RELU, scale_kind=oracle.SCALE_PER_COLUMN, reduce=reduce)
+    if reduce == oracle.RED_SOFTMAX:
+        np.testing.assert_allclose(Y.ravel(), _golden("softmax"), rtol=0, atol=1e-15)
+    else:
+        np.testing.assert_array_equal(Y.ravel(), _golden("y"))
+        np.testing.assert_allclose(out.ravel(), _golden(key), rtol=0, atol=1e-14)
+
+
+# ---------------------------------------------------------------- GEMM closed forms
+@pytest.mark.parametrize("act", [oracle.ACT_NONE, oracle.ACT_RELU])
+def test_identity_weights(act):
+    """W = I  =>  y = act(X + b) * s exactly."""
+    n = 24
+    X = _rand((5, n), 1)
+    b = gi.uniform(1, 3, n, -0.5, 0.5)
+    s = gi.uniform(1, 4, n, -1.5, 1.5)
+    Y, _, _ = _run(X, np.eye(n, dtype=np.float32), b, s, act=act, scale_kind=oracle.SCALE_PER_COLUMN,
+                   reduce=oracle.RED_MAXSUM)
+    u = X.astype(np.float64) + b.astype(np.float64)
+    if act == oracle.ACT_RELU:
+        u = np.maximum(u, 0)
+    np.testing.assert_array_equal(Y, u * s.astype(np.float64))
+
+
+def test_zero_weights_lse_is_log_n():
+    """W = 0, b = 0  =>  every y is 0, LSE = ln N, softmax = 1/N, (max, sum) = (0, 0)."""
+    M, N, K = 3, 40, 8
+    X, W = _rand((M, K), 2), np.zeros((N, K), np.float32)
+    _, out, _ = _run(X, W, None, None, act=oracle.ACT_GELU_TANH)
+    np.testing.assert_allclose(out[:, 0], math.log(N), rtol=0, atol=1e-15)
+    P, _, _ = _run(X, W, None, None, reduce=oracle.RED_SOFTMAX)
+    np.testing.assert_allclose(P, 1.0 / N, rtol=1e-15)
+    _, ms, _ = _run(X, W, None, None, reduce=oracle.RED_MAXSUM)
+    np.testing.assert_array_equal(ms, 0.0)
+
+
+def test_zero_weights_bias_only():
+    """W = 0  =>  y[m, n] = relu(b[n]) * s for every row."""
+    N = 16
+    b = gi.uniform(3, 3, N, -1, 1)
+    Y, out, _ = _run(_rand((4, 8), 3), np.zeros((N, 8), np.float32), b, None, act=oracle.ACT_RELU,
+                     scale_kind=oracle.SCALE_SCALAR, scale=-2.0, reduce=oracle.RED_MAXSUM)
+    ref = np.maximum(b.astype(np.float64), 0) * -2.0
+    np.testing.assert_array_equal(Y, np.tile(ref, (4, 1)))
+    np.testing.assert_array_equal(out[:, 0], ref.max())      # the max is taken after scaling
+    np.testing.assert_allclose(out[:, 1], ref.sum(), rtol=1e-15)
+
+
+def test_one_hot_rows_select_weight_columns():
+    """X[m, :] = e_j  =>  z[m, n] = W[n, j]; a transposed operand or swapped index fails this."""
+    M, N, K = 6, 10, 7
+    W = _rand((N, K), 4)
+    js = [0, 3, 6, 1, 5, 2]
+    X = np.zeros((M, K), np.float32)
+    X[np.arange(M), js] = 1
+    Y, _, _ = _run(X, W, None, None, reduce=oracle.RED_MAXSUM)
+    np.testing.assert_array_equal(Y, W[:, js].T.astype(np.float64))
+
+
+@pytest.mark.parametrize("dtype", [oracle.F32, oracle.BF16])
+def test_integer_inputs_are_exact(dtype):
+    """Small integers: every product and partial sum is an integer, so the result is exact."""
+    rng = np.random.default_rng(5)
+    B, M, N, K = 2, 9, 11, 33
+    Xi, Wi = rng.integers(-8, 9, (B, M, K)), rng.integers(-8, 9, (B, N, K))
+    bi = rng.integers(-4, 5, (B, N))
+    X, W = Xi.astype(np.float32), Wi.astype(np.float32)
+    if dtype == oracle.BF16:
+        X, W = gi.f32_to_bf16_bits(X).reshape(X.shape), gi.f32_to_bf16_bits(W).reshape(W.shape)
+    Y, out, _ = _run(X, W, bi.astype(np.float32), None, dtype=dtype, reduce=oracle.RED_MAXSUM, bias_per_batch=1)
+    Z = np.einsum("bmk,bnk->bmn", Xi, Wi) + bi[:, None, :]
+    np.testing.assert_array_equal(Y.reshape(B, M, N), Z.astype(np.float64))
+    np.testing.assert_array_equal(out.reshape(B, M, 2)[..., 0], Z.max(-1))
+    np.testing.assert_array_equal(out.reshape(B, M, 2)[..., 1], Z.sum(-1))
+
+
+def test_brute_force_4x4x4_rational():
+    """4x4x4 in exact rational arithmetic (ReLU, per-column scale, max+sum), then float LSE."""
+    X, W = _rand((4, 4), 6), _rand((4, 4), 6, tid=8)
+    b, s = gi.uniform(6, 3, 4, -1, 1), gi.uniform(6, 4, 4, 0.5, 1.5)
+    fx = [[Fraction(float(v)) for v in r] for r in X]
+    fw = [[Fraction(float(v)) for v in r] for r in W]
+    fy = [[max(sum(fx[m][k] * fw[n][k] for k in range(4)) + Fraction(float(b[n])), 0) * Fraction(float(s[n]))
+           for n in range(4)] for m in range(4)]
+    Y, ms, _ = _run(X, W, b, s, act=oracle.ACT_RELU, scale_kind=oracle.SCALE_PER_COLUMN, reduce=oracle.RED_MAXSUM)
+    for m in range(4):
+        for n in range(4):
+            assert abs(Y[m, n] - float(fy[m][n])) <= 4 * np.spacing(abs(float(fy[m][n])) + 1e-300)
+        assert ms[m, 0] == Y[m].max()
+        assert abs(ms[m, 1] - float(sum(fy[m]))) < 1e-15
+    _, lse, _ = _run(X, W, b, s, act=oracle.ACT_RELU, scale_kind=oracle.SCALE_PER_COLUMN, reduce=oracle.RED_LSE)
+    for m in range(4):
+        direct = math.log(math.fsum(math.exp(float(v)) for v in fy[m]))   # no max subtraction needed here
+        assert abs(lse[m, 0] - direct) < 1e-14
+
+
+# ---------------------------------------------------------------- GELU (tanh form)
+def test_gelu_symmetry_limits_monotone():
+    assert oracle.gelu_tanh(0.0) == 0.0
+    for x in [1e-3, 0.1, 0.5, 1.0, 2.5, 7.0]:
+        assert abs(oracle.gelu_tanh(x) - oracle.gelu_tanh(-x) - x) < 1e-15 * max(1, x)   # tanh is odd
+    assert oracle.gelu_tanh(8.0) == pytest.approx(8.0, abs=1e-12)
+    assert abs(oracle.gelu_tanh(-8.0)) < 1e-12
+    xs = np.linspace(0, 6, 200)
+    g = np.array([oracle.gelu_tanh(x) for x in xs])
+    assert np.all(np.diff(g) > 0)
+
+
+def test_gelu_against_decimal_arithmetic():
+    """The same function evaluated with 40-digit decimal exponentials (pins the two constants)."""
+    getcontext().prec = 40
+    pi = Decimal("3.14159265358979323846264338327950288420")
+    c = (Decimal(2) / pi).sqrt()
+    for x in ["-3.25", "-1", "-0.3", "0.2", "1", "1.7", "4.5"]:
+        u = Decimal(x)
+        t = c * (u + Decimal("0.044715") * u ** 3)
+        e2 = (2 * t).exp()
+        ref = Decimal("0.5") * u * (1 + (e2 - 1) / (e2 + 1))
+        assert abs(oracle.gelu_tanh(float(x)) - float(ref)) < 2e-16 * max(1.0, abs(float(ref)))
+
+
+def test_gelu_against_library():
+    xs = torch.linspace(-6, 6, 97, dtype=torch.float64)
+    ref = torch.nn.functional.gelu(xs, approximate="tanh").numpy()
+    got = np.array([oracle.act(oracle.ACT_GELU_TANH, float(x)) for x in xs])
+    np.testing.assert_allclose(got, ref, rtol=0, atol=2e-15)
+    assert oracle.act(oracle.ACT_RELU, -2.0) == 0.0 and oracle.act(oracle.ACT_RELU, 2.0) == 2.0
+    assert oracle.act(oracle.ACT_NONE, -2.0) == -2.0
+
+
+# ---------------------------------------------------------------- the whole chain vs library routines
+def _torch_chain(X, W, b, s_vec, act, scale_kind, scale, reduce, bias_per_batch):
+    X, W = torch.as_tensor(X, dtype=torch.float64), torch.as_tensor(W, dtype=torch.float64)
+    z = torch.matmul(X, W.transpose(-1, -2))
+    if b is not None:
+        bb = torch.as_tensor(b, dtype=torch.float64)
+        z = z + (bb.reshape(X.shape[0], 1, -1) if bias_per_batch else bb)
+    if act == oracle.ACT_RELU:
+        z = torch.relu(z)
+    elif act == oracle.ACT_GELU_TANH:
+        z = torch.nn.functional.gelu(z, approximate="tanh")
+    if scale_kind == oracle.SCALE_SCALAR:
+        z = z * scale
+    elif scale_kind == oracle.SCALE_PER_COLUMN:
+        z = z * torch.as_tensor(s_vec, dtype=torch.float64)
+    y = z.reshape(-1, z.shape[-1])
+    if reduce == oracle.RED_LSE:
+        return y, torch.logsumexp(y, 1, keepdim=True)
+    if reduce == oracle.RED_SOFTMAX:
+        return torch.softmax(y, 1), None
+    mx = y.amax(1, keepdim=True)
+    if reduce == oracle.RED_MAXSUM:
+        return y, torch.cat([mx, y.sum(1, keepdim=True)], 1)
+    return y, torch.cat([mx, torch.exp(y - mx).sum(1, keepdim=True)], 1)
+
+
+@pytest.mark.parametrize("dtype", [oracle.F32, oracle.BF16])
+@pytest.mark.parametrize("act", [0, 1, 2])
+@pytest.mark.parametrize("scale_kind", [0, 1, 2])
+@pytest.mark.parametrize("reduce", [0, 1, 2, 3])
+def test_against_fp64_library_chain(dtype, act, scale_kind, reduce):
+    B, M, N, K = 2, 7, 19, 13
+    seed = 100 + 16 * act + 4 * scale_kind + reduce
+    Xf, Wf = _rand((B, M, K), seed, std=1.5), _rand((B, N, K), seed, tid=8, std=1.5)
+    if dtype == oracle.BF16:
+        X, W = gi.f32_to_bf16_bits(Xf).reshape(Xf.shape), gi.f32_to_bf16_bits(Wf).reshape(Wf.shape)
+        Xf, Wf = gi.bf16_bits_to_f32(X).reshape(Xf.shape), gi.bf16_bits_to_f32(W).reshape(Wf.shape)
+    else:
+        X, W = Xf, Wf
+    b = gi.uniform(seed, 3, B * N, -1, 1)
+    s = gi.uniform(seed, 4, N, -1.5, 1.5)
+    Y, out, _ = oracle.run(X, W, b, s, dtype=dtype, act=act, scale_kind=scale_kind, reduce=reduce, scale=0.37,
+                           bias_per_batch=1)
+    ry, rout = _torch_chain(Xf, Wf, b, s, act, scale_kind, 0.37, reduce, 1)
+    np.testing.assert_allclose(Y, ry.numpy(), rtol=1e-12, atol=1e-13)
+    if rout is not None:
+        np.testing.assert_allclose(out, rout.numpy(), rtol=1e-12, atol=1e-13)
+
+
+def test_row_subset_and_batch_indexing():
+    p = gi.make_problem("t", 3, 5, 8, 16, gi.DTYPE_BF16, gi.ACT_GELU_TANH, gi.SCALE_SCALAR, gi.RED_LSE, scale=0.5, seed=9)
+    Yall, oall, _ = oracle.run_problem(p)
+    rows = np.array([14, 0, 7, 7, 3])
+    Y, o, _ = oracle.run_problem(p, rows=rows, nthreads=2)
+    np.testing.assert_array_equal(Y, Yall[rows])
+    np.testing.assert_array_equal(o, oall[rows])
+    Y1, o1, t1 = oracle.run_problem(p, nthreads=1)
+    assert t1 == 1
+    np.testing.assert_array_equal(Y1, Yall)      # independent of the thread count
+    with pytest.raises(ValueError):
+        oracle.run_problem(p, rows=[15])
+
+
+# ---------------------------------------------------------------- reductions: invariants
+def test_lse_bounds_shift_and_ties_between_kinds():
+    M, N, K = 9, 50, 12
+    X, W, b = _rand((M, K), 11, std=2.0), _rand((N, K), 11, tid=8, std=2.0), gi.uniform(11, 3, N, -1, 1)
+    Y, lse, _ = _run(X, W, b, None, reduce=oracle.RED_LSE)
+    mx = Y.max(1)
+    assert np.all(lse[:, 0] >= mx) and np.all(lse[:, 0] <= mx + math.log(N) + 1e-12)
+    _, lse_shift, _ = _run(X, W, b + np.float32(2.0), None, reduce=oracle.RED_LSE)   # b + 2 is exact in fp32 here? compare loosely
+    np.testing.assert_allclose(lse_shift[:, 0], lse[:, 0] + 2.0, rtol=0, atol=5e-7)
+    _, mse, _ = _run(X, W, b, None, reduce=oracle.RED_MAX_SUMEXP)
+    np.testing.assert_array_equal(mse[:, 0], mx)
+    assert np.all(mse[:, 1] >= 1.0) and np.all(mse[:, 1] <= N)
+    np.testing.assert_allclose(mse[:, 0] + np.log(mse[:, 1]), lse[:, 0], rtol=0, atol=1e-14)
+    P, _, _ = _run(X, W, b, None, reduce=oracle.RED_SOFTMAX)
+    np.testing.assert_allclose(P.sum(1), 1.0, rtol=0, atol=1e-12)
+    assert P.min() >= 0 and P.max() <= 1
+    np.testing.assert_allclose(P, np.exp(Y - lse), rtol=1e-12)
+    assert np.array_equal(np.argsort(P, 1, kind="stable"), np.argsort(Y, 1, kind="stable"))
+
+
+def test_lse_all_equal_row_and_large_logits():
+    """Equal logits: LSE = y + ln N.  Logits of +-800 (exp overflows in fp64 without the max shift)."""
+    N, K = 32, 4
+    X = np.ones((1, K), np.float32)
+    W = np.full((N, K), 0.25, np.float32)          # z = 1 for every n
+    _, lse, _ = _run(X, W, None, None, scale_kind=oracle.SCALE_SCALAR, scale=800.0)
+    assert lse[0, 0] == pytest.approx(800.0 + math.log(N), abs=1e-12)
+    _, lse, _ = _run(X, W, None, None, scale_kind=oracle.SCALE_SCALAR, scale=-800.0)
+    assert lse[0, 0] == pytest.approx(-800.0 + math.log(N), abs=1e-12)
+    W[5] = 0.5                                      # one dominant column: z = 2 -> 1600 vs 800
+    P, _, _ = _run(X, W, None, None, scale_kind=oracle.SCALE_SCALAR, scale=800.0, reduce=oracle.RED_SOFTMAX)
+    assert P[0, 5] == 1.0 and P[0].sum() == 1.0
+
+
+def test_maxsum_row_sum_is_a_gemv():
+    """act = NONE, s = 1:  sum_n y[m, n] = X[m, :] . (sum_n W[n, :]) + sum(b)."""
+    M, N, K = 8, 30, 20
+    X, W, b = _rand((M, K), 13), _rand((N, K), 13, tid=8), gi.uniform(13, 3, N, -1, 1)
+    _, ms, _ = _run(X, W, b, None, reduce=oracle.RED_MAXSUM)
+    ref = X.astype(np.float64) @ W.astype(np.float64).sum(0) + b.astype(np.float64).sum()
+    np.testing.assert_allclose(ms[:, 1], ref, rtol=0, atol=1e-13)
+    _, ms_relu, _ = _run(X, W, b, None, act=oracle.ACT_RELU, reduce=oracle.RED_MAXSUM)
+    assert np.all(ms_relu >= 0)
+
+
+def test_negative_scale_flips_the_max():
+    M, N, K = 4, 12, 6
+    X, W = _rand((M, K), 14), _rand((N, K), 14, tid=8)
+    Y, ms, _ = _run(X, W, None, None, reduce=oracle.RED_MAXSUM)
+    _, msn, _ = _run(X, W, None, None, scale_kind=oracle.SCALE_SCALAR, scale=-1.0, reduce=oracle.RED_MAXSUM)
+    np.testing.assert_array_equal(msn[:, 0], -Y.min(1))
+    np.testing.assert_allclose(msn[:, 1], -ms[:, 1], rtol=1e-15)
+
+
+def test_bad_arguments_are_rejected():
+    X, W = _rand((2, 4), 15), _rand((3, 4), 15, tid=8)
+    with pytest.raises(ValueError):
+        _run(X, W, None, None, scale_kind=oracle.SCALE_PER_COLUMN)      # needs a vector
+    with pytest.raises(TypeError):
+        _run(X.astype(np.float64), W, None, None)
+    with pytest.raises(ValueError):
+        _run(X, _rand((3, 5), 15), None, None)
