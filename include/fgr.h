@@ -1,0 +1,190 @@
+/*
+ * fgr.h - C ABI of the fused GEMM + epilogue + row-reduce operator for NVIDIA B200 (sm_100a).
+ *
+ * The operator.  For every batch bt and row m
+ *
+ *     z[m, n] = sum_k X[bt, m, k] * W[bt, n, k]            (X * W^T, K contiguous in both)
+ *     y[m, n] = act(z[m, n] + b[n]) * s[n]                  act in {identity, ReLU, GELU-tanh}
+ *
+ * followed by a reduction over n of each row:
+ *
+ *     FGR_RED_LSE        out[m]    = log sum_n exp(y[m, n])
+ *     FGR_RED_SOFTMAX    P[m, n]   = exp(y[m, n]) / sum_n exp(y[m, n])      (written in Y's slot)
+ *     FGR_RED_MAXSUM     out[m, :] = ( max_n y , sum_n y )
+ *     FGR_RED_MAX_SUMEXP out[m, :] = ( max_n y , sum_n exp(y - max_n y) )
+ *
+ * Where this comes from.  The paper's task statement is: given the reference operator's inputs,
+ * produce the same outputs, faster (Section 3.1, Verifier; Section 3.3), for operators of the
+ * categories "matrix multiplication, element-wise and reduction" (Section 1; Section 4.1,
+ * Datasets).  The paper prints no formula for any operator; the formulas above are the plain
+ * definitions of a linear layer, the activation, a scale and a last-dimension reduction.
+ *
+ * Conventions for every entry point.
+ *   - All functions return an fgr_status (0 = success) unless stated; nothing throws or aborts.
+ *   - "device pointer" = memory of the CUDA device named in the descriptor; "host pointer" =
+ *     ordinary process memory.  The caller owns every buffer it passes; the library owns only
+ *     the handle.  fgr_run never allocates and never synchronises.
+ *   - Layout: row-major.  X [batch, M, K], W [batch, N, K], Y / P [batch, M, N]; row strides
+ *     ldx, ldw, ldy and batch strides bsx, bsw, bsy in elements (0 = packed).
+ *   - Element types: X, W, Y/P are `dtype` (fp32, or bf16 as raw 16-bit patterns); bias,
+ *     scale_vec and out are always fp32.  Accumulation is fp32.
+ *   - Supported shapes: batch, M, N, K >= 1; K and N multiples of 8 (bf16) or 4 (fp32);
+ *     X, W, Y base pointers 16-byte aligned; ld* and bs* multiples of 8 (bf16) / 4 (fp32).
+ *     Anything else returns FGR_ERR_UNSUPPORTED or FGR_ERR_INVALID_ARG, never a wrong answer.
+ *   - Inputs must be finite.  NaN/Inf inputs give unspecified values but never hang or fault.
+ *   - One handle may be used by one thread and one stream at a time.
+ */
+#ifndef FGR_H_
+#define FGR_H_
+
+#if defined(__GNUC__)
+#define FGR_API __attribute__((visibility("default")))
+#else
+#define FGR_API
+#endif
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  FGR_OK = 0,
+  FGR_ERR_INVALID_ARG = 1,    /* null / misaligned pointer, bad enum, bad stride, bad struct size */
+  FGR_ERR_UNSUPPORTED = 2,    /* a shape the kernels do not cover (see "Supported shapes") */
+  FGR_ERR_WORKSPACE = 3,      /* workspace null, misaligned or smaller than fgr_workspace_bytes */
+  FGR_ERR_CUDA = 4,           /* a CUDA runtime/driver call failed (no device, launch error, ...) */
+  FGR_ERR_DEVICE_TIMEOUT = 5, /* a bounded in-kernel wait ran out; outputs of that run are invalid */
+  FGR_ERR_ARCH = 6            /* the device is not compute capability 10.x */
+} fgr_status;
+
+typedef enum { FGR_F32 = 0, FGR_BF16 = 1 } fgr_dtype;
+typedef enum { FGR_ACT_NONE = 0, FGR_ACT_RELU = 1, FGR_ACT_GELU_TANH = 2 } fgr_act;
+typedef enum { FGR_SCALE_NONE = 0, FGR_SCALE_SCALAR = 1, FGR_SCALE_PER_COLUMN = 2 } fgr_scale_kind;
+typedef enum { FGR_RED_LSE = 0, FGR_RED_SOFTMAX = 1, FGR_RED_MAXSUM = 2, FGR_RED_MAX_SUMEXP = 3 } fgr_reduce;
+
+/* Execution paths (fgr_plan_info.path, fgr_desc.force_path). */
+typedef enum {
+  FGR_PATH_AUTO = 0,
+  FGR_PATH_SIMT = 1,          /* CUDA-core tiles, fp32 FMA: the fp32 path, also valid for bf16 */
+  FGR_PATH_UMMA_TILED = 2,    /* tcgen05 128 x 256 tiles, TMA ring, compute-bound shapes (bf16) */
+  FGR_PATH_UMMA_STREAM_W = 3, /* tcgen05 with narrow N tiles and a deep TMA ring: M <= 128, W streamed once (bf16) */
+  FGR_PATH_SIMT_GEMV = 4      /* M <= 16: one warp per W row, 128-bit loads, shuffle reductions (bf16) */
+} fgr_path;
+
+typedef struct fgr_desc {
+  uint32_t struct_bytes;   /* = sizeof(fgr_desc) */
+  int32_t batch, M, N, K;
+  int32_t dtype;           /* fgr_dtype of X, W and Y/P */
+  int32_t act;             /* fgr_act */
+  int32_t scale_kind;      /* fgr_scale_kind */
+  int32_t reduce;          /* fgr_reduce */
+  float scale;             /* the scalar s when scale_kind == FGR_SCALE_SCALAR */
+  int32_t write_y;         /* 1: also write y to Y (SOFTMAX always writes P to Y) */
+  int64_t ldx, ldw, ldy;   /* row strides in elements; 0 = packed (K, K, N) */
+  int64_t bsx, bsw, bsy;   /* batch strides in elements; 0 = packed (M*ldx, N*ldw, M*ldy) */
+  int32_t bias_per_batch;  /* 0: bias[N] shared by all batches; 1: bias[batch, N] */
+  int32_t device;          /* CUDA device ordinal */
+  int32_t force_path;      /* fgr_path; FGR_PATH_AUTO lets the shape decide */
+  int32_t force_tile_n;    /* 0 = automatic; else the N extent of a tcgen05 tile (multiple of 16, 16..256) */
+} fgr_desc;
+
+/* What fgr_plan / fgr_create decided; plain host data, for callers, tests and benchmarks. */
+typedef struct fgr_plan_info {
+  int32_t path;            /* fgr_path actually used */
+  int32_t tile_m, tile_n;  /* output tile of one CTA */
+  int32_t stages;          /* depth of the shared-memory operand ring (0 for SIMT paths) */
+  int32_t parts_per_row;   /* number of split-N partial pairs per row in the workspace */
+  int32_t grid;            /* CTAs of the main kernel */
+  int32_t launches;        /* kernels launched by one fgr_run */
+  int32_t smem_bytes;      /* dynamic shared memory of the main kernel */
+  int64_t num_tiles;       /* output tiles in the problem */
+  uint64_t workspace_bytes;/* what fgr_run needs */
+  double flop;             /* 2 * batch * M * N * K */
+  double min_bytes;        /* operands read once + outputs written once */
+} fgr_plan_info;
+
+typedef struct fgr_handle fgr_handle; /* opaque */
+
+/*
+ * fgr_plan: validates a descriptor and reports path, tiling and workspace size.  Pure host
+ * arithmetic: touches no device, so it works without a GPU.  `num_sms` is the SM count to
+ * size the grid for (<= 0: 148).  This is the shape -> path selection: arithmetic intensity
+ * 2MNK / bytes against the machine's flop/byte ridge decides between the compute-bound tiled
+ * path and the weight-streaming path; dtype and M pick the SIMT paths.  (The paper's
+ * counterpart is the Conductor's bottleneck classification from profile metrics, Section 3.1;
+ * here it is a deterministic host rule.)
+ */
+FGR_API int fgr_plan(const fgr_desc* desc /*host*/, int num_sms, fgr_plan_info* info /*host, out*/);
+
+/*
+ * fgr_create: fgr_plan + device checks (the device must be compute capability 10.x, else
+ * FGR_ERR_ARCH) + kernel attribute set-up.  *out receives a handle that the caller frees with
+ * fgr_destroy.  No device memory is allocated.
+ */
+FGR_API int fgr_create(const fgr_desc* desc /*host*/, fgr_handle** out /*host, out*/);
+
+/* Bytes of device workspace fgr_run needs (>= 256; 0 if h is NULL).  Contents need no initialisation. */
+FGR_API size_t fgr_workspace_bytes(const fgr_handle* h);
+
+/* Copies the plan of a handle into *info. */
+FGR_API int fgr_get_plan(const fgr_handle* h, fgr_plan_info* info /*host, out*/);
+
+/*
+ * fgr_run: enqueues the whole operator (GEMM mainloop, fused epilogue, per-tile row reduction,
+ * split-N merge, softmax normalisation) on `cuda_stream` and returns without synchronising.
+ *   X, W       device, dtype, read-only
+ *   bias       device fp32 [N] (or [batch, N]); NULL = no bias
+ *   scale_vec  device fp32 [N]; required iff scale_kind == FGR_SCALE_PER_COLUMN
+ *   Y          device, dtype, [batch, M, N]; required iff write_y or SOFTMAX
+ *   out        device fp32: [batch*M] (LSE) or [batch*M, 2] (MAXSUM, MAX_SUMEXP); NULL for SOFTMAX
+ *   workspace  device, 256-byte aligned, at least fgr_workspace_bytes(h); scratch for the
+ *              split-N partial pairs and the device status word.  Two runs that overlap in time
+ *              must not share a workspace.
+ *   cuda_stream  a cudaStream_t passed as void*; NULL = the default stream
+ * Results are bit-identical from run to run (the merge order is fixed; no floating atomics).
+ */
+FGR_API int fgr_run(fgr_handle* h, const void* X, const void* W, const float* bias, const float* scale_vec,
+            void* Y, float* out, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * fgr_run_host: the same operator on HOST buffers (same shapes; packed or strided exactly as the
+ * descriptor says).  Copies the inputs to device staging buffers owned by the handle (allocated on
+ * the first call, freed by fgr_destroy), runs, copies Y / out back and synchronises before
+ * returning.  Returns the device status as fgr_get_status would.  Pinned host memory makes the
+ * copies asynchronous and faster but is not required.
+ */
+FGR_API int fgr_run_host(fgr_handle* h, const void* X, const void* W, const float* bias, const float* scale_vec,
+                 void* Y, float* out);
+
+/*
+ * fgr_get_status: synchronises the stream of the last fgr_run and returns the device status
+ * word: FGR_OK, or FGR_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel gave up (the kernels
+ * never trap and never spin without a limit), or FGR_ERR_CUDA if the stream reports an error.
+ */
+FGR_API int fgr_get_status(fgr_handle* h);
+
+/*
+ * Timing of the main kernel (the GEMM + epilogue + per-tile reduction launch), for benchmarks.
+ * fgr_profile_enable(h, 1): from now on fgr_run records a CUDA event before and after its main
+ * kernel on the run's stream (at most 4096 runs are kept; later runs are not recorded).
+ * fgr_profile_read synchronises those events, returns the summed main-kernel time in
+ * milliseconds and the number of runs it covers, and forgets them.  Off by default; this follows
+ * the timing protocol of Section 4.1 (Metrics): warm-up runs, then repeated timed runs.
+ */
+FGR_API int fgr_profile_enable(fgr_handle* h, int enable);
+FGR_API int fgr_profile_read(fgr_handle* h, double* main_kernel_ms /*host, out*/, int* runs /*host, out*/);
+
+/* Frees the handle and any staging memory it owns.  NULL is a no-op. */
+FGR_API int fgr_destroy(fgr_handle* h);
+
+/* Static strings; never NULL. */
+FGR_API const char* fgr_status_string(int status);
+FGR_API const char* fgr_path_name(int path);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FGR_H_ */

@@ -1,0 +1,479 @@
+// Host side of the fgr library: descriptor validation, shape -> path selection, tiling and
+// workspace layout, TMA descriptor encoding, and the extern "C" entry points of include/fgr.h.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "fgr_internal.h"
+
+using namespace fgr;
+
+struct fgr_handle {
+  fgr_desc desc;
+  fgr_plan_info plan;
+  Params base;               // everything but the per-run pointers
+  int num_sms;
+  // cached TMA descriptors (tcgen05 paths)
+  CUtensorMap tmap_x, tmap_w;
+  const void* cached_x;
+  const void* cached_w;
+  // status plumbing
+  void* last_workspace;
+  cudaStream_t last_stream;
+  bool ran;
+  // staging owned by the handle (fgr_run_host only)
+  void* stage[7];
+  size_t stage_bytes[7];
+  cudaStream_t host_stream;
+  // optional timing of the main kernel
+  bool profiling;
+  std::vector<cudaEvent_t>* events;   // pairs (before, after)
+  size_t events_used;
+};
+
+namespace {
+
+// Machine balance used by the selector: measured dense bf16 rate over measured HBM bandwidth of a
+// B200 (about 1640 TFLOP/s over about 6.5 TB/s), in flop per byte.
+constexpr double kRidgeFlopPerByte = 250.0;
+constexpr int kDefaultSms = 148;
+
+int elem_bytes(int dtype) { return dtype == FGR_F32 ? 4 : 2; }
+int out_width(int reduce) { return reduce == FGR_RED_LSE ? 1 : reduce == FGR_RED_SOFTMAX ? 0 : 2; }
+
+struct Resolved { long long ldx, ldw, ldy, bsx, bsw, bsy; };
+
+Resolved resolve_strides(const fgr_desc& d) {
+  Resolved r;
+  r.ldx = d.ldx ? d.ldx : d.K;
+  r.ldw = d.ldw ? d.ldw : d.K;
+  r.ldy = d.ldy ? d.ldy : d.N;
+  r.bsx = d.bsx ? d.bsx : (long long)d.M * r.ldx;
+  r.bsw = d.bsw ? d.bsw : (long long)d.N * r.ldw;
+  r.bsy = d.bsy ? d.bsy : (long long)d.M * r.ldy;
+  return r;
+}
+
+int validate(const fgr_desc* d) {
+  if (!d) return FGR_ERR_INVALID_ARG;
+  if (d->struct_bytes != sizeof(fgr_desc)) return FGR_ERR_INVALID_ARG;
+  if (d->dtype != FGR_F32 && d->dtype != FGR_BF16) return FGR_ERR_INVALID_ARG;
+  if (d->act < FGR_ACT_NONE || d->act > FGR_ACT_GELU_TANH) return FGR_ERR_INVALID_ARG;
+  if (d->scale_kind < FGR_SCALE_NONE || d->scale_kind > FGR_SCALE_PER_COLUMN) return FGR_ERR_INVALID_ARG;
+  if (d->reduce < FGR_RED_LSE || d->reduce > FGR_RED_MAX_SUMEXP) return FGR_ERR_INVALID_ARG;
+  if (d->force_path < FGR_PATH_AUTO || d->force_path > FGR_PATH_SIMT_GEMV) return FGR_ERR_INVALID_ARG;
+  if (d->batch < 1 || d->M < 1 || d->N < 1 || d->K < 1) return FGR_ERR_INVALID_ARG;
+  if (d->write_y != 0 && d->write_y != 1) return FGR_ERR_INVALID_ARG;
+  if (d->bias_per_batch != 0 && d->bias_per_batch != 1) return FGR_ERR_INVALID_ARG;
+  if (d->device < 0) return FGR_ERR_INVALID_ARG;
+  if (d->scale_kind == FGR_SCALE_SCALAR && !std::isfinite(d->scale)) return FGR_ERR_INVALID_ARG;
+  if (d->ldx < 0 || d->ldw < 0 || d->ldy < 0 || d->bsx < 0 || d->bsw < 0 || d->bsy < 0) return FGR_ERR_INVALID_ARG;
+  const int g = 16 / elem_bytes(d->dtype);   // elements per 16 bytes
+  if (d->K % g || d->N % g) return FGR_ERR_UNSUPPORTED;
+  const Resolved r = resolve_strides(*d);
+  if (r.ldx < d->K || r.ldw < d->K || r.ldy < d->N) return FGR_ERR_INVALID_ARG;
+  if (r.ldx % g || r.ldw % g || r.ldy % g || r.bsx % g || r.bsw % g || r.bsy % g) return FGR_ERR_UNSUPPORTED;
+  if (d->batch > 1 && (r.bsx < (long long)(d->M - 1) * r.ldx + d->K || r.bsw < (long long)(d->N - 1) * r.ldw + d->K ||
+                       r.bsy < (long long)(d->M - 1) * r.ldy + d->N))
+    return FGR_ERR_INVALID_ARG;
+  if ((long long)d->batch * d->M > (1LL << 31) - 1) return FGR_ERR_UNSUPPORTED;
+  if (d->force_tile_n && (d->force_tile_n % 16 || d->force_tile_n < 16 || d->force_tile_n > 256)) return FGR_ERR_INVALID_ARG;
+  return FGR_OK;
+}
+
+double min_bytes(const fgr_desc& d) {
+  const double e = elem_bytes(d.dtype);
+  double b = (double)d.batch * ((double)d.M * d.K + (double)d.N * d.K) * e;
+  b += 4.0 * d.N * (d.bias_per_batch ? d.batch : 1);   // bias (counted whether or not one is passed)
+  if (d.scale_kind == FGR_SCALE_PER_COLUMN) b += 4.0 * d.N;
+  if (d.write_y || d.reduce == FGR_RED_SOFTMAX) b += (double)d.batch * d.M * d.N * e;
+  b += 4.0 * d.batch * d.M * out_width(d.reduce);
+  return b;
+}
+
+// Narrow-tile choice for the weight-streaming path: every SM should stream an equal share of W
+// exactly once.  Cost model per wave: the W tile (tile_n rows) from HBM plus the X tile (128 rows)
+// from L2, per k-block.
+int pick_stream_tile_n(long long tiles_mb, int N, int sms) {
+  int best = 16;
+  double best_cost = 1e300;
+  for (int tn = 16; tn <= 256; tn += 16) {
+    const long long tiles = tiles_mb * ((N + tn - 1) / tn);
+    const long long waves = (tiles + sms - 1) / sms;
+    const double cost = (double)waves * (tn + 64);
+    if (cost < best_cost - 1e-9 || (std::fabs(cost - best_cost) <= 1e-9 && tn > best)) { best_cost = cost; best = tn; }
+  }
+  return best;
+}
+
+int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
+  const int sms = num_sms > 0 ? num_sms : kDefaultSms;
+  const Resolved r = resolve_strides(d);
+  fgr_plan_info pi;
+  std::memset(&pi, 0, sizeof pi);
+  pi.flop = 2.0 * d.batch * (double)d.M * d.N * d.K;
+  pi.min_bytes = min_bytes(d);
+
+  int path = d.force_path;
+  if (path == FGR_PATH_AUTO) {
+    if (d.dtype == FGR_F32) path = FGR_PATH_SIMT;
+    else if (d.M <= 128 && pi.flop / pi.min_bytes < kRidgeFlopPerByte) path = FGR_PATH_UMMA_STREAM_W;
+    else path = FGR_PATH_UMMA_TILED;
+  }
+  if (path == FGR_PATH_SIMT_GEMV) return FGR_ERR_UNSUPPORTED;   // not built yet
+  if ((path == FGR_PATH_UMMA_TILED || path == FGR_PATH_UMMA_STREAM_W) && d.dtype != FGR_BF16) return FGR_ERR_UNSUPPORTED;
+
+  Params p;
+  std::memset(&p, 0, sizeof p);
+  p.batch = d.batch; p.M = d.M; p.N = d.N; p.K = d.K;
+  p.dtype = d.dtype; p.act = d.act; p.scale_kind = d.scale_kind; p.reduce = d.reduce;
+  p.write_y = d.write_y; p.bias_per_batch = d.bias_per_batch; p.scale = d.scale;
+  p.ldx = r.ldx; p.ldw = r.ldw; p.ldy = r.ldy; p.bsx = r.bsx; p.bsw = r.bsw; p.bsy = r.bsy;
+
+  if (path == FGR_PATH_SIMT) {
+    p.tile_n = kSimtTile;
+    p.half_n = kSimtTile;
+    p.slots_per_tile = 1;
+    p.tiles_m = (d.M + kSimtTile - 1) / kSimtTile;
+    p.tiles_n = (d.N + kSimtTile - 1) / kSimtTile;
+    p.stages = 0;
+    pi.tile_m = kSimtTile;
+    pi.smem_bytes = 0;
+    if (p.tiles_m > 65535 || d.batch > 65535) return FGR_ERR_UNSUPPORTED;
+  } else {
+    p.tiles_m = (d.M + kUmmaTileM - 1) / kUmmaTileM;
+    int tn = d.force_tile_n;
+    if (!tn) {
+      if (path == FGR_PATH_UMMA_STREAM_W) tn = pick_stream_tile_n((long long)d.batch * p.tiles_m, d.N, sms);
+      else tn = d.N >= 256 ? 256 : ((d.N + 15) / 16) * 16;
+    }
+    p.tile_n = tn;
+    p.half_n = ((tn / 2 + 15) / 16) * 16;
+    p.slots_per_tile = 2;
+    p.tiles_n = (d.N + tn - 1) / tn;
+    int stages = kUmmaMaxStages;
+    while (stages > 1 && umma_smem_layout(tn, stages).total > kSmemLimit) --stages;
+    p.stages = stages;
+    pi.tile_m = kUmmaTileM;
+    pi.smem_bytes = umma_smem_layout(tn, stages).total;
+  }
+  p.num_tiles = (long long)d.batch * p.tiles_m * p.tiles_n;
+  p.parts_per_row = p.tiles_n * p.slots_per_tile;
+  if (d.reduce == FGR_RED_SOFTMAX && p.parts_per_row > 12288) return FGR_ERR_UNSUPPORTED;
+
+  pi.path = path;
+  pi.tile_n = p.tile_n;
+  pi.stages = p.stages;
+  pi.parts_per_row = p.parts_per_row;
+  pi.num_tiles = p.num_tiles;
+  pi.grid = path == FGR_PATH_SIMT ? (int)(p.num_tiles > 0x7fffffff ? 0x7fffffff : p.num_tiles)
+                                  : (int)(p.num_tiles < sms ? p.num_tiles : sms);
+  pi.launches = 2;   // main kernel + (merge | softmax normalise)
+  pi.workspace_bytes = (uint64_t)kStatusBytes + (uint64_t)d.batch * d.M * p.parts_per_row * 8ull;
+  *info = pi;
+  if (pp) *pp = p;
+  return FGR_OK;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(sym);
+  }
+  return fn;
+}
+
+// bf16 [batch, rows, K] with strides (ld, bs) -> 3-D map, box = 64 (K) x box_rows x 1, 128-byte swizzle,
+// out-of-range elements read as zero.
+int encode_operand(CUtensorMap* map, const void* ptr, int K, int rows, int batch, long long ld, long long bs, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return FGR_ERR_CUDA;
+  cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)batch};
+  cuuint64_t strides[2] = {(cuuint64_t)ld * 2, (cuuint64_t)(batch > 1 ? bs : (long long)rows * ld) * 2};
+  cuuint32_t box[3] = {(cuuint32_t)kUmmaBlockK, (cuuint32_t)box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS ? FGR_OK : FGR_ERR_CUDA;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+int fgr_plan(const fgr_desc* desc, int num_sms, fgr_plan_info* info) {
+  if (!info) return FGR_ERR_INVALID_ARG;
+  int rc = validate(desc);
+  if (rc != FGR_OK) return rc;
+  return make_plan(*desc, num_sms, info, nullptr);
+}
+
+int fgr_create(const fgr_desc* desc, fgr_handle** out) {
+  if (!out) return FGR_ERR_INVALID_ARG;
+  *out = nullptr;
+  int rc = validate(desc);
+  if (rc != FGR_OK) return rc;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || desc->device >= ndev) { cudaGetLastError(); return FGR_ERR_CUDA; }
+  int major = 0, sms = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, desc->device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, desc->device) != cudaSuccess)
+    return FGR_ERR_CUDA;
+  if (major != 10) return FGR_ERR_ARCH;
+  fgr_handle* h = new (std::nothrow) fgr_handle;
+  if (!h) return FGR_ERR_INVALID_ARG;
+  std::memset(h, 0, sizeof *h);
+  h->events = new (std::nothrow) std::vector<cudaEvent_t>();
+  if (!h->events) { delete h; return FGR_ERR_INVALID_ARG; }
+  h->desc = *desc;
+  h->num_sms = sms;
+  rc = make_plan(*desc, sms, &h->plan, &h->base);
+  if (rc != FGR_OK) { delete h->events; delete h; return rc; }
+  if (h->plan.path == FGR_PATH_UMMA_TILED || h->plan.path == FGR_PATH_UMMA_STREAM_W) {
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaError_t e = cudaSetDevice(desc->device);
+    if (e == cudaSuccess) e = umma_prepare(desc->device);
+    cudaSetDevice(prev);
+    if (e != cudaSuccess || !encode_fn()) { cudaGetLastError(); delete h->events; delete h; return FGR_ERR_CUDA; }
+  }
+  *out = h;
+  return FGR_OK;
+}
+
+size_t fgr_workspace_bytes(const fgr_handle* h) { return h ? (size_t)h->plan.workspace_bytes : 0; }
+
+int fgr_get_plan(const fgr_handle* h, fgr_plan_info* info) {
+  if (!h || !info) return FGR_ERR_INVALID_ARG;
+  *info = h->plan;
+  return FGR_OK;
+}
+
+int fgr_run(fgr_handle* h, const void* X, const void* W, const float* bias, const float* scale_vec, void* Y,
+            float* out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!h || !X || !W) return FGR_ERR_INVALID_ARG;
+  const fgr_desc& d = h->desc;
+  const bool softmax = d.reduce == FGR_RED_SOFTMAX;
+  if (!aligned16(X) || !aligned16(W) || (Y && !aligned16(Y))) return FGR_ERR_INVALID_ARG;
+  if ((d.write_y || softmax) && !Y) return FGR_ERR_INVALID_ARG;
+  if (!softmax && !out) return FGR_ERR_INVALID_ARG;
+  if (d.scale_kind == FGR_SCALE_PER_COLUMN && !scale_vec) return FGR_ERR_INVALID_ARG;
+  if ((bias && (reinterpret_cast<uintptr_t>(bias) & 3u)) || (scale_vec && (reinterpret_cast<uintptr_t>(scale_vec) & 3u)) ||
+      (out && (reinterpret_cast<uintptr_t>(out) & 7u)))
+    return FGR_ERR_INVALID_ARG;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < h->plan.workspace_bytes)
+    return FGR_ERR_WORKSPACE;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+  int prev = -1;
+  cudaGetDevice(&prev);
+  if (prev != d.device && cudaSetDevice(d.device) != cudaSuccess) { cudaGetLastError(); return FGR_ERR_CUDA; }
+  int rc = FGR_OK;
+  cudaError_t e = cudaSuccess;
+
+  Params p = h->base;
+  p.X = X; p.W = W; p.bias = bias; p.scale_vec = scale_vec; p.Y = Y; p.out = out;
+  p.status = static_cast<int*>(workspace);
+  p.parts = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes);
+
+  if (workspace != h->last_workspace) {   // a workspace seen for the first time: clear its status word
+    e = cudaMemsetAsync(workspace, 0, kStatusBytes, stream);
+    h->last_workspace = workspace;
+  }
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  if (h->profiling && h->events_used + 2 <= 2 * 4096) {
+    if (h->events->size() < h->events_used + 2) {
+      cudaEvent_t a = nullptr, b = nullptr;
+      if (cudaEventCreate(&a) == cudaSuccess && cudaEventCreate(&b) == cudaSuccess) { h->events->push_back(a); h->events->push_back(b); }
+    }
+    if (h->events->size() >= h->events_used + 2) { ev0 = (*h->events)[h->events_used]; ev1 = (*h->events)[h->events_used + 1]; }
+  }
+  if (e == cudaSuccess && ev0) e = cudaEventRecord(ev0, stream);
+  if (e == cudaSuccess) {
+    if (h->plan.path == FGR_PATH_SIMT) {
+      e = launch_simt(p, stream);
+    } else {
+      if (X != h->cached_x) {
+        rc = encode_operand(&h->tmap_x, X, d.K, d.M, d.batch, p.ldx, p.bsx, kUmmaTileM);
+        h->cached_x = rc == FGR_OK ? X : nullptr;
+      }
+      if (rc == FGR_OK && W != h->cached_w) {
+        rc = encode_operand(&h->tmap_w, W, d.K, d.N, d.batch, p.ldw, p.bsw, p.tile_n);
+        h->cached_w = rc == FGR_OK ? W : nullptr;
+      }
+      if (rc == FGR_OK) e = launch_umma(p, &h->tmap_x, &h->tmap_w, h->plan.grid, h->plan.smem_bytes, stream);
+    }
+  }
+  if (rc == FGR_OK && e == cudaSuccess && ev1) {
+    e = cudaEventRecord(ev1, stream);
+    h->events_used += 2;
+  }
+  if (rc == FGR_OK && e == cudaSuccess) e = softmax ? launch_normalise(p, stream) : launch_merge(p, stream);
+  if (e != cudaSuccess) { cudaGetLastError(); rc = FGR_ERR_CUDA; }
+  h->last_stream = stream;
+  h->ran = true;
+  if (prev != d.device && prev >= 0) cudaSetDevice(prev);
+  return rc;
+}
+
+int fgr_get_status(fgr_handle* h) {
+  if (!h) return FGR_ERR_INVALID_ARG;
+  if (!h->ran) return FGR_OK;
+  int prev = -1;
+  cudaGetDevice(&prev);
+  if (prev != h->desc.device) cudaSetDevice(h->desc.device);
+  int word = 0;
+  int rc = FGR_OK;
+  if (cudaStreamSynchronize(h->last_stream) != cudaSuccess ||
+      cudaMemcpy(&word, h->last_workspace, sizeof word, cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    rc = FGR_ERR_CUDA;
+  } else if (word != 0) {
+    rc = word;
+    cudaMemset(h->last_workspace, 0, sizeof word);   // reported once
+  }
+  if (prev != h->desc.device && prev >= 0) cudaSetDevice(prev);
+  return rc;
+}
+
+int fgr_run_host(fgr_handle* h, const void* X, const void* W, const float* bias, const float* scale_vec, void* Y,
+                 float* out) {
+  if (!h || !X || !W) return FGR_ERR_INVALID_ARG;
+  const fgr_desc& d = h->desc;
+  const Params& b = h->base;
+  const bool softmax = d.reduce == FGR_RED_SOFTMAX;
+  const bool need_y = d.write_y || softmax;
+  if ((need_y && !Y) || (!softmax && !out)) return FGR_ERR_INVALID_ARG;
+  if (d.scale_kind == FGR_SCALE_PER_COLUMN && !scale_vec) return FGR_ERR_INVALID_ARG;
+  const size_t e = (size_t)elem_bytes(d.dtype);
+  // extents in bytes of each buffer as laid out by the descriptor's strides
+  const size_t want[7] = {
+      ((size_t)(d.batch - 1) * b.bsx + (size_t)(d.M - 1) * b.ldx + d.K) * e,
+      ((size_t)(d.batch - 1) * b.bsw + (size_t)(d.N - 1) * b.ldw + d.K) * e,
+      bias ? (size_t)d.N * (d.bias_per_batch ? d.batch : 1) * 4 : 0,
+      scale_vec ? (size_t)d.N * 4 : 0,
+      need_y ? ((size_t)(d.batch - 1) * b.bsy + (size_t)(d.M - 1) * b.ldy + d.N) * e : 0,
+      (size_t)d.batch * d.M * out_width(d.reduce) * 4,
+      (size_t)h->plan.workspace_bytes};
+  int prev = -1;
+  cudaGetDevice(&prev);
+  if (prev != d.device && cudaSetDevice(d.device) != cudaSuccess) { cudaGetLastError(); return FGR_ERR_CUDA; }
+  int rc = FGR_OK;
+  if (!h->host_stream && cudaStreamCreateWithFlags(&h->host_stream, cudaStreamNonBlocking) != cudaSuccess) rc = FGR_ERR_CUDA;
+  for (int i = 0; i < 7 && rc == FGR_OK; ++i) {
+    if (want[i] > h->stage_bytes[i]) {
+      if (h->stage[i]) cudaFree(h->stage[i]);
+      h->stage[i] = nullptr;
+      h->stage_bytes[i] = 0;
+      if (cudaMalloc(&h->stage[i], want[i]) != cudaSuccess) rc = FGR_ERR_CUDA;
+      else h->stage_bytes[i] = want[i];
+      if (i == 0) h->cached_x = nullptr;   // a new allocation may reuse an old address with other strides
+      if (i == 1) h->cached_w = nullptr;
+    }
+  }
+  cudaStream_t s = h->host_stream;
+  const void* src[4] = {X, W, bias, scale_vec};
+  for (int i = 0; i < 4 && rc == FGR_OK; ++i)
+    if (want[i] && cudaMemcpyAsync(h->stage[i], src[i], want[i], cudaMemcpyHostToDevice, s) != cudaSuccess) rc = FGR_ERR_CUDA;
+  if (rc == FGR_OK)
+    rc = fgr_run(h, h->stage[0], h->stage[1], bias ? static_cast<float*>(h->stage[2]) : nullptr,
+                 scale_vec ? static_cast<float*>(h->stage[3]) : nullptr, need_y ? h->stage[4] : nullptr,
+                 softmax ? nullptr : static_cast<float*>(h->stage[5]), h->stage[6], h->stage_bytes[6], s);
+  if (rc == FGR_OK && need_y && cudaMemcpyAsync(Y, h->stage[4], want[4], cudaMemcpyDeviceToHost, s) != cudaSuccess) rc = FGR_ERR_CUDA;
+  if (rc == FGR_OK && want[5] && !softmax &&
+      cudaMemcpyAsync(out, h->stage[5], want[5], cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    rc = FGR_ERR_CUDA;
+  if (rc == FGR_OK) rc = fgr_get_status(h);
+  else cudaGetLastError();
+  if (prev != d.device && prev >= 0) cudaSetDevice(prev);
+  return rc;
+}
+
+int fgr_profile_enable(fgr_handle* h, int enable) {
+  if (!h) return FGR_ERR_INVALID_ARG;
+  h->profiling = enable != 0;
+  return FGR_OK;
+}
+
+int fgr_profile_read(fgr_handle* h, double* main_kernel_ms, int* runs) {
+  if (!h || !main_kernel_ms || !runs) return FGR_ERR_INVALID_ARG;
+  double sum = 0.0;
+  int n = 0, rc = FGR_OK;
+  int prev = -1;
+  cudaGetDevice(&prev);
+  if (prev != h->desc.device) cudaSetDevice(h->desc.device);
+  for (size_t i = 0; i + 1 < h->events_used; i += 2) {
+    float ms = 0.0f;
+    if (cudaEventSynchronize((*h->events)[i + 1]) != cudaSuccess ||
+        cudaEventElapsedTime(&ms, (*h->events)[i], (*h->events)[i + 1]) != cudaSuccess) { cudaGetLastError(); rc = FGR_ERR_CUDA; break; }
+    sum += ms;
+    ++n;
+  }
+  if (prev != h->desc.device && prev >= 0) cudaSetDevice(prev);
+  h->events_used = 0;
+  *main_kernel_ms = sum;
+  *runs = n;
+  return rc;
+}
+
+int fgr_destroy(fgr_handle* h) {
+  if (!h) return FGR_OK;
+  bool owns = h->host_stream != nullptr || !h->events->empty();
+  for (int i = 0; i < 7; ++i) owns = owns || h->stage[i];
+  if (owns) {
+    int prev = -1;
+    cudaGetDevice(&prev);
+    if (prev != h->desc.device) cudaSetDevice(h->desc.device);
+    if (h->host_stream) { cudaStreamSynchronize(h->host_stream); cudaStreamDestroy(h->host_stream); }
+    for (int i = 0; i < 7; ++i) if (h->stage[i]) cudaFree(h->stage[i]);
+    for (cudaEvent_t ev : *h->events) cudaEventDestroy(ev);
+    if (prev != h->desc.device && prev >= 0) cudaSetDevice(prev);
+  }
+  delete h->events;
+  delete h;
+  return FGR_OK;
+}
+
+const char* fgr_status_string(int status) {
+  switch (status) {
+    case FGR_OK: return "ok";
+    case FGR_ERR_INVALID_ARG: return "invalid argument";
+    case FGR_ERR_UNSUPPORTED: return "unsupported shape or configuration";
+    case FGR_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case FGR_ERR_CUDA: return "CUDA call failed";
+    case FGR_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    case FGR_ERR_ARCH: return "device is not compute capability 10.x";
+    default: return "unknown status";
+  }
+}
+
+const char* fgr_path_name(int path) {
+  switch (path) {
+    case FGR_PATH_AUTO: return "auto";
+    case FGR_PATH_SIMT: return "simt";
+    case FGR_PATH_UMMA_TILED: return "umma_tiled";
+    case FGR_PATH_UMMA_STREAM_W: return "umma_stream_w";
+    case FGR_PATH_SIMT_GEMV: return "simt_gemv";
+    default: return "unknown";
+  }
+}
+
+}  // extern "C"

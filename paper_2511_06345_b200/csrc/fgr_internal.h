@@ -1,0 +1,77 @@
+// Internal declarations shared by the host dispatcher and the kernels of the fgr library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "fgr.h"
+
+namespace fgr {
+
+constexpr int kStatusBytes = 256;     // head of the workspace: device status word + diagnostics
+constexpr int kUmmaTileM = 128;       // rows of one tcgen05 accumulator tile (= TMEM lanes)
+constexpr int kUmmaBlockK = 64;       // bf16 elements per K block = one 128-byte swizzle row
+constexpr int kUmmaThreads = 320;     // warp 0 TMA producer, warp 1 MMA issuer, warps 2..9 epilogue
+constexpr int kUmmaMaxStages = 12;
+constexpr int kSimtTile = 64;         // SIMT path: 64 x 64 output tile per CTA
+constexpr int kSmemLimit = 232448;    // 227 KB: the per-CTA opt-in maximum on sm_100
+
+// Kernel parameters: plain values and device pointers.
+struct Params {
+  int batch, M, N, K;
+  int dtype, act, scale_kind, reduce, write_y, bias_per_batch;
+  float scale;
+  long long ldx, ldw, ldy, bsx, bsw, bsy;
+  const void* X;
+  const void* W;
+  const float* bias;
+  const float* scale_vec;
+  void* Y;
+  float* out;
+  float* parts;        // [batch * M][parts_per_row][2] split-N partial pairs
+  int* status;         // device status word (0 = ok)
+  int parts_per_row;
+  int tile_n;          // N extent of one tile
+  int half_n;          // tcgen05 paths: columns [0, half_n) of a tile go to slot 0, the rest to slot 1
+  int slots_per_tile;  // partial pairs per (row, tile): 1 (SIMT) or 2 (tcgen05)
+  int tiles_m, tiles_n;
+  long long num_tiles;
+  int stages;
+};
+
+// Column -> partial-slot mapping shared by the producers of the partials and the normalise pass.
+__host__ __device__ inline int part_slot(int col, int tile_n, int half_n, int slots_per_tile) {
+  int t = col / tile_n;
+  int w = col - t * tile_n;
+  return t * slots_per_tile + ((slots_per_tile == 2 && w >= half_n) ? 1 : 0);
+}
+
+// Shared-memory carve-up of the tcgen05 kernel (offsets from a 1024-byte aligned base).
+struct UmmaSmem {
+  int stage_bytes, x_bytes, w_bytes;
+  int vec_off;      // bias / scale staging: [8 epilogue warps][2 vectors][128] floats
+  int bar_off;      // mbarriers
+  int misc_off;     // TMEM base address, abort flag
+  int total;        // bytes to request (includes 1024 of alignment slack)
+};
+__host__ __device__ inline UmmaSmem umma_smem_layout(int tile_n, int stages) {
+  UmmaSmem s;
+  s.x_bytes = kUmmaTileM * kUmmaBlockK * 2;
+  s.w_bytes = tile_n * kUmmaBlockK * 2;
+  s.stage_bytes = s.x_bytes + s.w_bytes;
+  s.vec_off = s.stage_bytes * stages;
+  s.bar_off = s.vec_off + 8 * 2 * 128 * 4;
+  s.misc_off = s.bar_off + (2 * kUmmaMaxStages + 4) * 8;
+  s.total = s.misc_off + 16 + 1024;
+  return s;
+}
+
+// Launchers (each enqueues on `stream` and returns the cudaError_t of the launch).
+cudaError_t launch_simt(const Params& p, cudaStream_t stream);
+cudaError_t launch_merge(const Params& p, cudaStream_t stream);
+cudaError_t launch_normalise(const Params& p, cudaStream_t stream);
+cudaError_t umma_prepare(int device);   // opt-in shared memory attribute, once per device
+cudaError_t launch_umma(const Params& p, const void* tmap_x, const void* tmap_w, int grid, int smem_bytes,
+                        cudaStream_t stream);
+
+}  // namespace fgr

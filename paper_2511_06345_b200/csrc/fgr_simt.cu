@@ -1,0 +1,277 @@
+// CUDA-core kernels of the fgr library:
+//   - simt_gemm_kernel: 64 x 64 output tiles, fp32 FMA, fused epilogue and per-tile row reduction
+//     (the fp32 path; also a valid path for bf16 inputs),
+//   - merge_kernel: combines the split-N partial pairs of every row in a fixed order,
+//   - normalise_kernel: second pass of the softmax (rescales the stored exponentials).
+// Accurate expf / logf / tanhf throughout: fp32 outputs are held to 1e-4 * (1 + |ref|).
+#include <cuda_bf16.h>
+#include <math_constants.h>
+
+#include "fgr_internal.h"
+
+namespace fgr {
+namespace {
+
+constexpr int BK = 16;
+constexpr int PAD = 4;
+
+__device__ __forceinline__ float4 load4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
+  uint2 r = *reinterpret_cast<const uint2*>(p);
+  float4 f;
+  f.x = __uint_as_float(r.x << 16);
+  f.y = __uint_as_float(r.x & 0xffff0000u);
+  f.z = __uint_as_float(r.y << 16);
+  f.w = __uint_as_float(r.y & 0xffff0000u);
+  return f;
+}
+__device__ __forceinline__ void store4(float* p, float a, float b, float c, float d) {
+  *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d);
+}
+__device__ __forceinline__ void store4(__nv_bfloat16* p, float a, float b, float c, float d) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+  uint2 r;
+  r.x = *reinterpret_cast<uint32_t*>(&lo);
+  r.y = *reinterpret_cast<uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(p) = r;
+}
+
+__device__ __forceinline__ float activation(int act, float u) {
+  if (act == FGR_ACT_RELU) return fmaxf(u, 0.0f);
+  if (act == FGR_ACT_GELU_TANH) {
+    const float c = 0.7978845608028654f;  // sqrt(2 / pi)
+    return 0.5f * u * (1.0f + tanhf(c * (u + 0.044715f * u * u * u)));
+  }
+  return u;
+}
+
+__device__ __forceinline__ float group16_max(float v) {
+#pragma unroll
+  for (int o = 8; o >= 1; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float group16_sum(float v) {
+#pragma unroll
+  for (int o = 8; o >= 1; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) simt_gemm_kernel(const Params p) {
+  __shared__ __align__(16) float Xs[BK][kSimtTile + PAD];
+  __shared__ __align__(16) float Ws[BK][kSimtTile + PAD];
+
+  const int bt = blockIdx.z;
+  const int m0 = blockIdx.y * kSimtTile;
+  const int n0 = blockIdx.x * kSimtTile;
+  const int t = threadIdx.x;
+  const int tx = t & 15, ty = t >> 4;
+  const int lr = t >> 2, lk = (t & 3) * 4;
+
+  const T* X = static_cast<const T*>(p.X) + (long long)bt * p.bsx;
+  const T* W = static_cast<const T*>(p.W) + (long long)bt * p.bsw;
+
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
+
+  for (int k0 = 0; k0 < p.K; k0 += BK) {
+    float4 xv = make_float4(0.f, 0.f, 0.f, 0.f), wv = xv;
+    if (k0 + lk < p.K) {   // K is a multiple of 4: the four elements are in range together
+      if (m0 + lr < p.M) xv = load4(X + (long long)(m0 + lr) * p.ldx + k0 + lk);
+      if (n0 + lr < p.N) wv = load4(W + (long long)(n0 + lr) * p.ldw + k0 + lk);
+    }
+    __syncthreads();
+    Xs[lk + 0][lr] = xv.x; Xs[lk + 1][lr] = xv.y; Xs[lk + 2][lr] = xv.z; Xs[lk + 3][lr] = xv.w;
+    Ws[lk + 0][lr] = wv.x; Ws[lk + 1][lr] = wv.y; Ws[lk + 2][lr] = wv.z; Ws[lk + 3][lr] = wv.w;
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < BK; ++k) {
+      float4 a = *reinterpret_cast<const float4*>(&Xs[k][ty * 4]);
+      float4 b = *reinterpret_cast<const float4*>(&Ws[k][tx * 4]);
+      const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+  }
+
+  // ---- fused epilogue: y = act(z + b) * s, in registers
+  const int nc = n0 + tx * 4;
+  const bool cols_ok = nc < p.N;   // N is a multiple of 4: the four columns are in range together
+  float bj[4] = {0.f, 0.f, 0.f, 0.f}, sj[4] = {1.f, 1.f, 1.f, 1.f};
+  if (cols_ok) {
+    if (p.bias) {
+      const float* b = p.bias + (p.bias_per_batch ? (long long)bt * p.N : 0);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) bj[j] = b[nc + j];
+    }
+    if (p.scale_kind == FGR_SCALE_PER_COLUMN) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) sj[j] = p.scale_vec[nc + j];
+    } else if (p.scale_kind == FGR_SCALE_SCALAR) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) sj[j] = p.scale;
+    }
+  }
+  T* Y = static_cast<T*>(p.Y) + (long long)bt * p.bsy;
+  const bool exp_kind = p.reduce != FGR_RED_MAXSUM;
+  const bool store_y = p.write_y && p.reduce != FGR_RED_SOFTMAX;
+
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int m = m0 + ty * 4 + i;
+    float y[4];
+    float mx = -CUDART_INF_F, sm = 0.0f;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      y[j] = activation(p.act, acc[i][j] + bj[j]) * sj[j];
+      if (cols_ok) { mx = fmaxf(mx, y[j]); sm += y[j]; }
+    }
+    if (store_y && cols_ok && m < p.M) store4(Y + (long long)m * p.ldy + nc, y[0], y[1], y[2], y[3]);
+    // ---- per-tile row reduction across the 16 threads that share this row
+    mx = group16_max(mx);
+    float second;
+    if (exp_kind) {
+      float e[4], l = 0.0f;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { e[j] = cols_ok ? expf(y[j] - mx) : 0.0f; l += e[j]; }
+      if (p.reduce == FGR_RED_SOFTMAX && cols_ok && m < p.M)
+        store4(Y + (long long)m * p.ldy + nc, e[0], e[1], e[2], e[3]);
+      second = group16_sum(l);
+    } else {
+      second = group16_sum(sm);
+    }
+    if (tx == 0 && m < p.M) {
+      float2* dst = reinterpret_cast<float2*>(p.parts) +
+                    ((long long)bt * p.M + m) * p.parts_per_row + blockIdx.x;
+      *dst = make_float2(mx, second);
+    }
+  }
+}
+
+// One warp per row: lane t takes partials t, t + 32, ... in ascending order, then a fixed
+// xor-shuffle tree combines the 32 lanes.  The order never depends on timing: bit-identical
+// results from run to run.
+__global__ void __launch_bounds__(256) merge_kernel(const Params p) {
+  const long long row = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= (long long)p.batch * p.M) return;
+  const float2* src = reinterpret_cast<const float2*>(p.parts) + row * p.parts_per_row;
+  const bool exp_kind = p.reduce != FGR_RED_MAXSUM;
+  float a = -CUDART_INF_F, b = 0.0f;
+  for (int t = lane; t < p.parts_per_row; t += 32) {
+    float2 v = src[t];
+    if (exp_kind) {
+      float mn = fmaxf(a, v.x);
+      if (mn > -CUDART_INF_F) b = b * expf(a - mn) + v.y * expf(v.x - mn);
+      a = mn;
+    } else {
+      a = fmaxf(a, v.x);
+      b += v.y;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) {
+    float oa = __shfl_xor_sync(0xffffffffu, a, o), ob = __shfl_xor_sync(0xffffffffu, b, o);
+    if (exp_kind) {
+      float mn = fmaxf(a, oa);
+      // both operands of the sum are evaluated in the same (lower lane first) order on both lanes
+      float lo_a = (lane & o) ? oa : a, lo_b = (lane & o) ? ob : b;
+      float hi_a = (lane & o) ? a : oa, hi_b = (lane & o) ? b : ob;
+      b = (mn > -CUDART_INF_F) ? lo_b * expf(lo_a - mn) + hi_b * expf(hi_a - mn) : 0.0f;
+      a = mn;
+    } else {
+      float lo_b = (lane & o) ? ob : b, hi_b = (lane & o) ? b : ob;
+      a = fmaxf(a, oa);
+      b = lo_b + hi_b;
+    }
+  }
+  if (lane == 0) {
+    if (p.reduce == FGR_RED_LSE) p.out[row] = a + logf(b);
+    else if (p.reduce != FGR_RED_SOFTMAX) reinterpret_cast<float2*>(p.out)[row] = make_float2(a, b);
+  }
+}
+
+// Softmax, second pass.  The GEMM pass stored E[m, n] = exp(y - m_slot) per partial slot together
+// with (m_slot, l_slot).  One CTA per row: the first warp merges the slots into (m_row, l_row) and
+// leaves the factor exp(m_slot - m_row) / l_row of every slot in shared memory; then the CTA
+// rescales the row with 16-byte accesses.
+template <typename T>
+__global__ void __launch_bounds__(256) normalise_kernel(const Params p) {
+  extern __shared__ float factor[];   // [parts_per_row]
+  const long long row = blockIdx.x;
+  const int bt = (int)(row / p.M), m = (int)(row % p.M);
+  const float2* src = reinterpret_cast<const float2*>(p.parts) + row * p.parts_per_row;
+  if (threadIdx.x < 32) {
+    const int lane = threadIdx.x;
+    float a = -CUDART_INF_F;
+    for (int t = lane; t < p.parts_per_row; t += 32) a = fmaxf(a, src[t].x);
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+    float l = 0.0f;
+    for (int t = lane; t < p.parts_per_row; t += 32) {
+      float2 v = src[t];
+      float f = (v.x > -CUDART_INF_F) ? expf(v.x - a) : 0.0f;
+      factor[t] = f;
+      l += v.y * f;
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+      float ol = __shfl_xor_sync(0xffffffffu, l, o);
+      l = (lane & o) ? ol + l : l + ol;
+    }
+    const float inv = 1.0f / l;
+    for (int t = lane; t < p.parts_per_row; t += 32) factor[t] *= inv;
+  }
+  __syncthreads();
+  T* y = static_cast<T*>(p.Y) + (long long)bt * p.bsy + (long long)m * p.ldy;
+  constexpr int V = 16 / (int)sizeof(T);   // elements per 16-byte access; N is a multiple of V
+  for (int c = threadIdx.x * V; c < p.N; c += blockDim.x * V) {
+    uint4 raw = *reinterpret_cast<const uint4*>(y + c);
+    if constexpr (sizeof(T) == 4) {
+      float* f = reinterpret_cast<float*>(&raw);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) f[j] *= factor[part_slot(c + j, p.tile_n, p.half_n, p.slots_per_tile)];
+    } else {
+      uint32_t* w = reinterpret_cast<uint32_t*>(&raw);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        float lo = __uint_as_float(w[j] << 16), hi = __uint_as_float(w[j] & 0xffff0000u);
+        lo *= factor[part_slot(c + 2 * j, p.tile_n, p.half_n, p.slots_per_tile)];
+        hi *= factor[part_slot(c + 2 * j + 1, p.tile_n, p.half_n, p.slots_per_tile)];
+        __nv_bfloat162 r = __floats2bfloat162_rn(lo, hi);
+        w[j] = *reinterpret_cast<uint32_t*>(&r);
+      }
+    }
+    *reinterpret_cast<uint4*>(y + c) = raw;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_simt(const Params& p, cudaStream_t stream) {
+  dim3 grid((unsigned)p.tiles_n, (unsigned)p.tiles_m, (unsigned)p.batch);
+  if (p.dtype == FGR_F32) simt_gemm_kernel<float><<<grid, 256, 0, stream>>>(p);
+  else simt_gemm_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_merge(const Params& p, cudaStream_t stream) {
+  const long long rows = (long long)p.batch * p.M;
+  merge_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_normalise(const Params& p, cudaStream_t stream) {
+  const long long rows = (long long)p.batch * p.M;
+  const size_t smem = (size_t)p.parts_per_row * sizeof(float);
+  if (p.dtype == FGR_F32) normalise_kernel<float><<<(unsigned)rows, 256, smem, stream>>>(p);
+  else normalise_kernel<__nv_bfloat16><<<(unsigned)rows, 256, smem, stream>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace fgr

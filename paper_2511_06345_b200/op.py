@@ -1,0 +1,62 @@
+"""Convenience wrapper over the C ABI for torch users: allocates outputs and workspace with torch
+and passes raw pointers and the current stream to ``fgr_run``.  No arithmetic happens here."""
+from __future__ import annotations
+
+import torch
+
+from . import binding as B
+
+
+class FusedGemmReduce:
+    """One operator instance (a handle of the C library) bound to a CUDA device.
+
+    ``__call__(X, W, bias=None, scale_vec=None)`` returns ``(Y_or_None, out_or_None)``:
+    Y / P is bf16 or fp32 [batch, M, N]; out is fp32 [batch*M] (LSE) or [batch*M, 2].
+    X [batch, M, K] and W [batch, N, K] are packed CUDA tensors (bf16 or fp32 as configured).
+    """
+
+    def __init__(self, batch, M, N, K, dtype, act, scale_kind, reduce, *, scale=1.0, write_y=0, bias_per_batch=0,
+                 device=0, force_path=B.FGR_PATH_AUTO, force_tile_n=0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("a CUDA device is required: this operator has no CPU path")
+        self.desc = B.make_desc(batch, M, N, K, dtype, act, scale_kind, reduce, scale=scale, write_y=write_y,
+                                bias_per_batch=bias_per_batch, device=device, force_path=force_path,
+                                force_tile_n=force_tile_n)
+        self.handle = B.fgr_create(self.desc)
+        self.plan = B.fgr_get_plan(self.handle)
+        self.device = torch.device("cuda", device)
+        self.workspace_bytes = B.fgr_workspace_bytes(self.handle)
+        self.workspace = torch.empty(self.workspace_bytes, dtype=torch.uint8, device=self.device)
+        self.tdtype = torch.float32 if dtype == B.FGR_F32 else torch.bfloat16
+        rows = batch * M
+        self.need_y = bool(write_y) or reduce == B.FGR_RED_SOFTMAX
+        self.out_shape = None if reduce == B.FGR_RED_SOFTMAX else ((rows,) if reduce == B.FGR_RED_LSE else (rows, 2))
+
+    @property
+    def path(self) -> str:
+        return B.fgr_path_name(self.plan.path)
+
+    def __call__(self, X, W, bias=None, scale_vec=None, Y=None, out=None):
+        d = self.desc
+        if Y is None and self.need_y:
+            Y = torch.empty((d.batch, d.M, d.N), dtype=self.tdtype, device=self.device)
+        if out is None and self.out_shape is not None:
+            out = torch.empty(self.out_shape, dtype=torch.float32, device=self.device)
+        stream = torch.cuda.current_stream(self.device).cuda_stream
+        B.fgr_run(self.handle, X, W, bias, scale_vec, Y if self.need_y else None, out, self.workspace,
+                  self.workspace_bytes, stream)
+        return (Y if self.need_y else None), out
+
+    def status(self) -> int:
+        return B.fgr_get_status(self.handle)
+
+    def close(self):
+        if self.handle is not None:
+            B.fgr_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
