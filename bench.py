@@ -1,0 +1,356 @@
+#!/usr/bin/env python
+"""Benchmark of the fused GEMM + epilogue + row-reduce operator on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config c2] [--impl ours|reference]
+
+One step = one pass of the whole hot path (GEMM mainloop, fused epilogue, per-tile row reduction,
+split-N merge / softmax normalisation) over one seeded synthetic problem of the named workload.
+Rank 0 prints ONE JSON line.  With N > 1 (torchrun) every rank runs its own problem on its own GPU
+(rows/batches are independent: no collective on the data path; weak scaling).
+
+Timing: W warm-up steps, then K steps between two CUDA events on the launching stream, bracketed
+by a barrier and a device synchronise; max over ranks.  Consecutive steps use different input and
+output buffers (a rotation larger than the 126 MB L2), so no step finds its operands in L2.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+L2_BYTES = 126e6
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+METRIC = "fused GEMM+epilogue+rowreduce TFLOP/s (or GB/s) and % of roofline, 1 B200"
+HBM_BOUND = {"c4"}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the GPU works."""
+
+    def __init__(self, index: int, period_s: float = 0.005):
+        self.index, self.period = index, period_s
+        self.samples = []          # (host time, sm MHz, reasons bitmask)
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self.ok = False
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                try:
+                    reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    reasons = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                self.samples.append((time.perf_counter(), float(mhz), int(reasons)))
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.ok:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread:
+            self._stop.set()
+            self._thread.join()
+
+    def summary(self, t0: float, t1: float):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"], "samples": 0}
+        inside = [s for s in self.samples if t0 <= s[0] <= t1]
+        window = "timed region"
+        if len(inside) < 3:        # a very short region: fall back to everything sampled under load
+            inside, window = self.samples, "warm-up + timed region"
+        mhz = sorted(s[1] for s in inside)
+        bits = 0
+        for s in inside:
+            bits |= s[2]
+        names = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+                 0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+                 0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+        reasons = [n for b, n in names.items() if bits & b and n != "gpu_idle"]
+        return {"sm_mhz": mhz[len(mhz) // 2], "sm_max_mhz": self.max_mhz, "reasons": reasons,
+                "samples": len(inside), "window": window}
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def oracle_sample(p, seconds: float):
+    """Times the CPU oracle, as it stands, on a leading block of rows sized for about `seconds`."""
+    import numpy as np
+    import oracle
+    total = p.batch * p.M
+    probe = min(total, 16)
+    t = time.perf_counter()
+    _, _, threads = oracle.run_problem(p, rows=np.arange(probe), want_y=False)
+    dt = max(time.perf_counter() - t, 1e-4)
+    rows = int(max(probe, min(total, probe * seconds / dt)))
+    stride = max(1, total // rows)
+    idx = (np.arange(rows) * stride) % total
+    t = time.perf_counter()
+    oracle.run_problem(p, rows=idx, want_y=False)
+    dt = time.perf_counter() - t
+    flop = 2.0 * rows * p.N * p.K
+    return flop, dt, threads, rows
+
+
+def unit_and_value(cfg, p, seconds_per_step, n_problems=1):
+    if cfg in HBM_BOUND:
+        return "GB/s", n_problems * p.min_bytes() / seconds_per_step / 1e9
+    return "TFLOP/s", n_problems * p.flop / seconds_per_step / 1e12
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    import fgr_inputs as gi
+    p = gi.make_config(args.config, seed=0)
+    per_step = min(2.0, 60.0 / max(args.steps, 1))   # the whole run stays near a minute of CPU time
+    flop = dt = 0.0
+    threads = rows = 0
+    for _ in range(max(args.warmup, 0)):
+        oracle_sample(p, 0.2)
+    f_sum = t_sum = 0.0
+    for _ in range(args.steps):
+        flop, dt, threads, rows = oracle_sample(p, per_step)
+        f_sum += flop
+        t_sum += dt
+    if args.config in HBM_BOUND:
+        unit, value = "GB/s", (f_sum / p.flop) * p.min_bytes() / t_sum / 1e9
+    else:
+        unit, value = "TFLOP/s", f_sum / t_sum / 1e12
+    sample = "%d of %d rows per step (every %d-th row), all N and K" % (rows, p.batch * p.M, max(1, p.batch * p.M // rows))
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": unit, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * t_sum / max(args.steps, 1), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.config, "note": "CPU fp64 oracle on a bounded row sample"},
+        "cpu_baseline": {"value": value, "unit": unit, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    import fgr_inputs as gi
+    import paper_2511_06345_b200 as fgr
+
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the operator has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    cfg = args.config
+    peaks, peak_src = load_peaks()
+
+    sampler = ClockSampler(local_rank)
+    # ---- inputs: a rotation of distinct problems so that no step finds its operands in L2
+    shape = gi.make_config(cfg, materialize=False)
+    set_bytes = shape.min_bytes()
+    rot = max(2, int(math.ceil(2.4 * L2_BYTES / set_bytes)) + 1)
+    rot = min(rot, 8)
+    b16 = shape.dtype == gi.DTYPE_BF16
+    tdt = torch.bfloat16 if b16 else torch.float32
+
+    def up(a, bits16):
+        t = torch.from_numpy(np.ascontiguousarray(a))
+        if bits16:
+            t = t.view(torch.int16).view(torch.bfloat16)
+        return t.to(dev)
+
+    sets = []
+    host0 = None
+    for r in range(rot):
+        p = gi.make_config(cfg, seed=1000 * rank + r)
+        if r == 0:
+            host0 = p
+        sets.append(dict(X=up(p.X, b16), W=up(p.W, b16),
+                         bias=None if p.bias is None else up(p.bias, False),
+                         scale=None if p.scale_vec is None else up(p.scale_vec, False)))
+    p = host0
+    need_y = bool(p.write_y) or p.reduce == gi.RED_SOFTMAX
+    rows = p.batch * p.M
+    for s in sets:
+        s["Y"] = torch.empty((p.batch, p.M, p.N), dtype=tdt, device=dev) if need_y else None
+        s["out"] = torch.empty((rows, p.out_width), dtype=torch.float32, device=dev) if p.out_width else None
+
+    desc = fgr.make_desc(p.batch, p.M, p.N, p.K, p.dtype, p.act, p.scale_kind, p.reduce, scale=p.scale,
+                         write_y=p.write_y, bias_per_batch=p.bias_per_batch, device=local_rank)
+    h = fgr.fgr_create(desc)
+    plan = fgr.fgr_get_plan(h)
+    ws_bytes = fgr.fgr_workspace_bytes(h)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream(dev).cuda_stream
+
+    def step(i):
+        s = sets[i % rot]
+        fgr.fgr_run(h, s["X"], s["W"], s["bias"], s["scale"], s["Y"], s["out"], ws, ws_bytes, stream)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    sampler.start()
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+    fgr.fgr_profile_enable(h, True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_host0 = time.perf_counter()
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    barrier()
+    t_host1 = time.perf_counter()
+    sampler.stop()
+    fgr.fgr_profile_enable(h, False)
+    status = fgr.fgr_get_status(h)
+    if status != fgr.FGR_OK:
+        raise SystemExit("device status after the timed region: " + fgr.fgr_status_string(status))
+    ms_total = e0.elapsed_time(e1)
+    kern_ms, kern_runs = fgr.fgr_profile_read(h)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    unit, value = unit_and_value(cfg, p, ms_step * 1e-3, n_problems=world)
+    clocks = sampler.summary(t_host0, t_host1)
+
+    # ---- roofline of the dominant kernel (the main GEMM + epilogue launch)
+    kern_s = (kern_ms / max(kern_runs, 1)) * 1e-3
+    if cfg in HBM_BOUND:
+        roof = {"bound": "hbm", "achieved": p.min_bytes() / kern_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    else:
+        roof = {"bound": "tensor", "achieved": p.flop / kern_s / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac_of_sustained_peak": p.flop / kern_s / 1e12 / peaks["bf16_tflops_sustained"]}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["peak_source"] = peak_src + (" (burst)" if roof["bound"] == "tensor" else "")
+    roof["kernel"] = "umma_kernel" if plan.path in (fgr.FGR_PATH_UMMA_TILED, fgr.FGR_PATH_UMMA_STREAM_W) else "simt_gemm_kernel"
+    roof["kernel_us"] = kern_s * 1e6
+    roof["traffic"] = TRAFFIC.get(cfg)
+
+    # ---- end to end: host buffers through fgr_run_host, copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        hp = {k: (None if v is None else v.cpu().pin_memory()) for k, v in sets[0].items()}
+        e2e_steps = max(3, min(args.steps, 20))
+        for _ in range(2):
+            fgr.fgr_run_host(h, hp["X"], hp["W"], hp["bias"], hp["scale"], hp["Y"], hp["out"])
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            fgr.fgr_run_host(h, hp["X"], hp["W"], hp["bias"], hp["scale"], hp["Y"], hp["out"])
+        torch.cuda.synchronize(dev)
+        dt = (time.perf_counter() - t0) / e2e_steps
+        if world > 1:
+            import torch.distributed as dist
+            t = torch.tensor([dt], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        eu, ev = unit_and_value(cfg, p, dt, n_problems=world)
+        h2d = sum(hp[k].numel() * hp[k].element_size() for k in ("X", "W", "bias", "scale") if hp[k] is not None)
+        d2h = sum(hp[k].numel() * hp[k].element_size() for k in ("Y", "out") if hp[k] is not None)
+        e2e = {"value": ev, "unit": eu, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+               "ms_per_step": dt * 1e3}
+    fgr.fgr_destroy(h)
+
+    # ---- the CPU oracle timed beside it (rank 0, single-GPU runs only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        flop, dt, threads, nrows = oracle_sample(p, 12.0)
+        if cfg in HBM_BOUND:
+            cu, cv = "GB/s", (flop / p.flop) * p.min_bytes() / dt / 1e9
+        else:
+            cu, cv = "TFLOP/s", flop / dt / 1e12
+        cpu = {"value": cv, "unit": cu, "cores": threads, "kind": "oracle", "seconds": dt,
+               "sample": "%d of %d rows (evenly spaced), all N and K, fp64 triple loop" % (nrows, rows)}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if b16 else "f32", "data": "synthetic",
+            "config": {"workload": cfg, "batch": p.batch, "M": p.M, "N": p.N, "K": p.K,
+                       "act": ["none", "relu", "gelu_tanh"][p.act], "scale": ["none", "scalar", "per_column"][p.scale_kind],
+                       "reduce": ["lse", "softmax", "maxsum", "max_sumexp"][p.reduce], "write_y": int(need_y),
+                       "path": fgr.fgr_path_name(plan.path), "tile": [plan.tile_m, plan.tile_n], "stages": plan.stages,
+                       "grid": plan.grid, "l2": "rotating %d distinct input/output sets (%.0f MB > 126 MB L2)" % (rot, rot * set_bytes / 1e6),
+                       "parallelism": "independent problems per GPU, no collective" if world > 1 else "1 GPU"},
+            "clocks": clocks, "gpu_launches": args.steps * plan.launches, "roofline": roof,
+        }
+        if e2e is not None:
+            line["e2e"] = e2e
+        if cpu is not None:
+            line["cpu_baseline"] = cpu
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+# DRAM bytes per launch of the main kernel from ncu (dram__bytes_read.sum + dram__bytes_write.sum);
+# None until a capture of the current kernel exists.
+TRAFFIC = {}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

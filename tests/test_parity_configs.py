@@ -1,0 +1,87 @@
+"""GPU parity at the full sizes of the five named workloads, in the launch configuration the
+benchmark times.  Rows are independent, so the oracle evaluates a sample of rows exactly (all N
+columns of each); c1 and c4 are compared in full."""
+import numpy as np
+import pytest
+
+import fgr_inputs as gi
+import paper_2511_06345_b200 as fgr
+from parity import compare, run_gpu, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+def _rows(total, block, count, seed):
+    rng = np.random.default_rng(seed)
+    edge = [0, 1, block - 1, block, block + 1, total - block, total - 1, total // 2]
+    rnd = rng.choice(total, size=count, replace=False).tolist()
+    return np.array(sorted(set(r for r in edge + rnd if 0 <= r < total)), dtype=np.int64)
+
+
+def test_c1_full(cuda_device):
+    p = gi.make_config("c1")
+    Y, out, plan = run_gpu(p)
+    assert plan["path"] == fgr.FGR_PATH_SIMT
+    w = compare(p, Y, out, tcgen05=False)
+    assert w["out"] <= 1e-4
+
+
+@pytest.mark.parametrize("reduce", [gi.RED_MAXSUM, gi.RED_MAX_SUMEXP])
+def test_c2_sampled_rows(cuda_device, reduce):
+    p = gi.make_config("c2", reduce=reduce)
+    Y, out, plan = run_gpu(p)
+    assert plan["path"] == fgr.FGR_PATH_UMMA_TILED and plan["tile_n"] == 256 and plan["grid"] > 100
+    rows = _rows(p.M, 128, 40, 2)
+    w = compare(p, Y, out, rows=rows)
+    assert w["Y"] <= 2e-2 and w["out"] <= 2e-2
+    # properties that hold for every row: ReLU and positive scales -> max >= 0, sum >= 0, max <= sum
+    if reduce == gi.RED_MAXSUM:
+        assert (out[:, 0] >= 0).all() and (out[:, 1] >= out[:, 0] - 1e-3).all()
+        np.testing.assert_allclose(Y.max(1), out[:, 0], rtol=4e-3, atol=1e-6)     # bf16 Y vs fp32 max
+        np.testing.assert_allclose(Y.sum(1), out[:, 1], rtol=2e-3)
+
+
+def test_c3_softmax_sampled_rows(cuda_device):
+    p = gi.make_config("c3")
+    Y, out, plan = run_gpu(p)
+    assert out is None and plan["parts_per_row"] >= 2          # the split-N merge is exercised
+    rows = _rows(p.M, 128, 24, 3)
+    compare(p, Y, out, rows=rows)
+    s = Y.sum(1)
+    assert np.abs(s - 1).max() <= 1e-2 and Y.min() >= 0 and Y.max() <= 1
+
+
+def test_c3_shape_with_spread_logits(cuda_device):
+    """Same shape, but a scale that spreads the logits over +-25 so that the maximum subtraction and
+    the rescaling between tiles matter (at the workload's own scale every P is close to 1/N)."""
+    p = gi.make_config("c3", scale=8.0, M=1024)
+    Y, out, _ = run_gpu(p)
+    rows = _rows(p.M, 128, 16, 4)
+    compare(p, Y, out, rows=rows)
+    assert np.abs(Y.sum(1) - 1).max() <= 1e-2
+
+
+def test_c4_full(cuda_device):
+    p = gi.make_config("c4")
+    Y, out, plan = run_gpu(p)
+    assert plan["path"] == fgr.FGR_PATH_UMMA_STREAM_W and Y is None
+    assert 140 <= plan["num_tiles"] <= plan["grid"] + 0 or plan["num_tiles"] <= 148
+    w = compare(p, Y, out)
+    assert w["out"] <= 2e-2
+    pw = gi.make_config("c4", write_y=1)
+    Y, out, _ = run_gpu(pw, tensors=to_device(pw))
+    compare(pw, Y, out, rows=_rows(p.M, 64, 12, 5))
+
+
+@pytest.mark.parametrize("reduce", [gi.RED_MAXSUM, gi.RED_MAX_SUMEXP])
+def test_c5_batched_sampled_rows(cuda_device, reduce):
+    p = gi.make_config("c5", reduce=reduce)
+    Y, out, plan = run_gpu(p)
+    assert Y is None and plan["num_tiles"] == 1024
+    rows = _rows(p.batch * p.M, 1024, 48, 6)
+    compare(p, Y, out, rows=rows)
+    if reduce == gi.RED_MAXSUM:
+        assert (out >= 0).all()
+    pw = gi.make_config("c5", write_y=1, batch=4)
+    Y, out, _ = run_gpu(pw)
+    compare(pw, Y, out, rows=_rows(pw.batch * pw.M, 1024, 16, 7))
