@@ -167,6 +167,35 @@ FGR_API int fgr_run_host(fgr_handle* h, const void* X, const void* W, const floa
 FGR_API int fgr_get_status(fgr_handle* h);
 
 /*
+ * fgr_run_static: the same operator for callers that cannot allocate device memory.  (The paper has
+ * no counterpart; this is a deployment convenience.)
+ *
+ * Who needs it: code running where cudaMalloc is not an option - inside a framework whose caching
+ * allocator owns the device, in a latency-critical loop that must not take the allocator's locks,
+ * or in an embedding that is handed buffers but no allocator.  Such a caller cannot produce the
+ * workspace fgr_run asks for, and has no handle.  Here the split-N partial pairs live in a fixed
+ * array of FGR_STATIC_SCRATCH_BYTES inside the library image (each GPU that loads the library holds
+ * those bytes until the process exits); the caller passes only the descriptor, inputs and outputs.
+ * The call allocates nothing on the device or through any library, and creates no handle.
+ *
+ *   - Always uses the CUDA-core path (FGR_PATH_SIMT; force_path must be AUTO or SIMT), fp32 or bf16.
+ *     Results are those of fgr_run on that path.
+ *   - Size limit: batch * M * ceil(N / 64) * 8 bytes must fit in FGR_STATIC_SCRATCH_BYTES, else
+ *     FGR_ERR_WORKSPACE is returned and nothing is launched.
+ *   - X, W, bias, scale_vec, Y, out: device pointers with the meaning and alignment fgr_run requires.
+ *   - The first call on a device looks up the device address of the scratch array and checks the
+ *     architecture; make that first call outside any stream capture.  Later calls only launch.
+ *   - All calls on a device share the one array.  It keeps whatever the previous call left, which is
+ *     harmless: every pair the merge pass reads is written earlier in the same call, so nothing has
+ *     to be cleared.  Two calls whose kernels may overlap on the GPU (different streams, no ordering
+ *     between them) race on the array: order them, or use fgr_run with separate workspaces.
+ *   - Asynchronous on `cuda_stream`; launch errors come back as FGR_ERR_CUDA.
+ */
+#define FGR_STATIC_SCRATCH_BYTES (4u << 20)
+FGR_API int fgr_run_static(const fgr_desc* desc /*host*/, const void* X, const void* W, const float* bias,
+                           const float* scale_vec, void* Y, float* out, void* cuda_stream);
+
+/*
  * Timing of the main kernel (the GEMM + epilogue + per-tile reduction launch), for benchmarks.
  * fgr_profile_enable(h, 1): from now on fgr_run records a CUDA event before and after its main
  * kernel on the run's stream (at most 4096 runs are kept; later runs are not recorded).

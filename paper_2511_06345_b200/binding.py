@@ -19,7 +19,9 @@ FGR_SCALE_NONE, FGR_SCALE_SCALAR, FGR_SCALE_PER_COLUMN = 0, 1, 2
 FGR_RED_LSE, FGR_RED_SOFTMAX, FGR_RED_MAXSUM, FGR_RED_MAX_SUMEXP = 0, 1, 2, 3
 FGR_PATH_AUTO, FGR_PATH_SIMT, FGR_PATH_UMMA_TILED, FGR_PATH_UMMA_STREAM_W, FGR_PATH_SIMT_GEMV = 0, 1, 2, 3, 4
 
-EXPORTS = ("fgr_plan", "fgr_create", "fgr_workspace_bytes", "fgr_get_plan", "fgr_run", "fgr_run_host",
+FGR_STATIC_SCRATCH_BYTES = 4 << 20
+
+EXPORTS = ("fgr_plan", "fgr_create", "fgr_workspace_bytes", "fgr_get_plan", "fgr_run", "fgr_run_host", "fgr_run_static",
            "fgr_get_status", "fgr_profile_enable", "fgr_profile_read", "fgr_destroy", "fgr_status_string", "fgr_path_name")
 
 
@@ -68,6 +70,7 @@ def lib() -> ctypes.CDLL:
         L.fgr_get_plan.argtypes, L.fgr_get_plan.restype = [vp, ctypes.POINTER(fgr_plan_info)], i
         L.fgr_run.argtypes, L.fgr_run.restype = [vp] * 8 + [ctypes.c_size_t, vp], i
         L.fgr_run_host.argtypes, L.fgr_run_host.restype = [vp] * 7, i
+        L.fgr_run_static.argtypes, L.fgr_run_static.restype = [ctypes.POINTER(fgr_desc)] + [vp] * 7, i
         L.fgr_get_status.argtypes, L.fgr_get_status.restype = [vp], i
         L.fgr_profile_enable.argtypes, L.fgr_profile_enable.restype = [vp, i], i
         L.fgr_profile_read.argtypes, L.fgr_profile_read.restype = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i)], i
@@ -143,6 +146,17 @@ def fgr_run_host(h, X, W, bias, scale_vec, Y, out, check=True) -> int:
     rc = lib().fgr_run_host(h, _addr(X), _addr(W), _addr(bias), _addr(scale_vec), _addr(Y), _addr(out))
     if check and rc != FGR_OK:
         raise FgrError(rc, "fgr_run_host")
+    return rc
+
+
+def fgr_run_static(desc: fgr_desc, X, W, bias, scale_vec, Y, out, stream=None, check=True) -> int:
+    """The operator without a handle or workspace, for callers that cannot allocate device memory:
+    the scratch is a fixed array inside the library (see include/fgr.h for the size limit and the
+    sharing rules).  Device pointers (ints or tensors); ``stream`` a raw cudaStream_t value or None."""
+    rc = lib().fgr_run_static(ctypes.byref(desc), _addr(X), _addr(W), _addr(bias), _addr(scale_vec), _addr(Y),
+                              _addr(out), stream)
+    if check and rc != FGR_OK:
+        raise FgrError(rc, "fgr_run_static")
     return rc
 
 
