@@ -230,24 +230,35 @@ __global__ void __launch_bounds__(256) normalise_kernel(const Params p) {
   __syncthreads();
   T* y = static_cast<T*>(p.Y) + (long long)bt * p.bsy + (long long)m * p.ldy;
   constexpr int V = 16 / (int)sizeof(T);   // elements per 16-byte access; N is a multiple of V
-  for (int c = threadIdx.x * V; c < p.N; c += blockDim.x * V) {
-    uint4 raw = *reinterpret_cast<const uint4*>(y + c);
+  // Slot boundaries are multiples of 16 columns, so the V elements of one access share a factor.
+  auto scale_vec = [&](uint4 raw, float f) {
     if constexpr (sizeof(T) == 4) {
-      float* f = reinterpret_cast<float*>(&raw);
+      float* v = reinterpret_cast<float*>(&raw);
 #pragma unroll
-      for (int j = 0; j < 4; ++j) f[j] *= factor[part_slot(c + j, p.tile_n, p.half_n, p.slots_per_tile)];
+      for (int j = 0; j < 4; ++j) v[j] *= f;
     } else {
       uint32_t* w = reinterpret_cast<uint32_t*>(&raw);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        float lo = __uint_as_float(w[j] << 16), hi = __uint_as_float(w[j] & 0xffff0000u);
-        lo *= factor[part_slot(c + 2 * j, p.tile_n, p.half_n, p.slots_per_tile)];
-        hi *= factor[part_slot(c + 2 * j + 1, p.tile_n, p.half_n, p.slots_per_tile)];
-        __nv_bfloat162 r = __floats2bfloat162_rn(lo, hi);
+        __nv_bfloat162 r = __floats2bfloat162_rn(__uint_as_float(w[j] << 16) * f, __uint_as_float(w[j] & 0xffff0000u) * f);
         w[j] = *reinterpret_cast<uint32_t*>(&r);
       }
     }
-    *reinterpret_cast<uint4*>(y + c) = raw;
+    return raw;
+  };
+  const int stride = blockDim.x * V;
+  int c = threadIdx.x * V;
+  for (; c + stride < p.N; c += 2 * stride) {   // two independent 16-byte accesses in flight per thread
+    const uint4 a0 = *reinterpret_cast<const uint4*>(y + c);
+    const uint4 a1 = *reinterpret_cast<const uint4*>(y + c + stride);
+    const float f0 = factor[part_slot(c, p.tile_n, p.half_n, p.slots_per_tile)];
+    const float f1 = factor[part_slot(c + stride, p.tile_n, p.half_n, p.slots_per_tile)];
+    *reinterpret_cast<uint4*>(y + c) = scale_vec(a0, f0);
+    *reinterpret_cast<uint4*>(y + c + stride) = scale_vec(a1, f1);
+  }
+  if (c < p.N) {
+    const uint4 a0 = *reinterpret_cast<const uint4*>(y + c);
+    *reinterpret_cast<uint4*>(y + c) = scale_vec(a0, factor[part_slot(c, p.tile_n, p.half_n, p.slots_per_tile)]);
   }
 }
 

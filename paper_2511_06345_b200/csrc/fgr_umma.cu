@@ -1,393 +1,29 @@
-// tcgen05 path of the fgr library (bf16 inputs, fp32 accumulation in tensor memory).
-//
-// One persistent CTA per SM, 10 warps with fixed roles:
-//   warp 0      TMA producer: X and W k-blocks (64 bf16 = one 128-byte swizzled row per matrix row)
-//               into a ring of shared-memory stages, completion on "full" mbarriers;
-//   warp 1      MMA issuer: one thread issues tcgen05.mma (128 x tile_n x 16 per instruction) into
-//               one of two TMEM accumulator buffers; tcgen05.commit releases ring stages ("empty")
-//               and publishes finished accumulators ("tmem_full");
-//   warps 2..9  epilogue: tcgen05.ld of the accumulator (thread = one output row, 32 TMEM lanes per
-//               warp, two warps share a lane quadrant and split the tile's columns), bias +
-//               activation + scale in registers, running row reduction, optional bf16 store, one
-//               partial pair per (row, tile half) to the workspace, then "tmem_empty".
-// The epilogue of tile i overlaps the mainloop of tile i + 1 through the two accumulator buffers.
-//
-// Every mbarrier wait is bounded: after about a second it records FGR_ERR_DEVICE_TIMEOUT in the
-// device status word, raises a CTA-wide abort flag that all other waits observe, and the CTA drains
-// (waits, bounded, for TMA copies still in flight), frees its tensor memory and returns.
-#include <cuda.h>
-#include <cuda_bf16.h>
-#include <math_constants.h>
-
-#include "fgr_internal.h"
+// Dispatch of the tcgen05 path: picks the compiled kernel variant for a problem's activation,
+// scaling, reduction kind and Y store.  The kernel itself is in fgr_umma_kernel.cuh.
+#include "fgr_umma_kernel.cuh"
 
 namespace fgr {
-namespace {
-
-constexpr uint32_t kTmemCols = 512;
-constexpr int kChunk = 16;                       // accumulator columns per tcgen05.ld
-constexpr long long kWaitCycles = 2000000000LL;  // about one second at ~2 GHz
-
-// ------------------------------------------------------------------------------------------ PTX
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.b32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-
-// Bounded wait.  Returns false if the CTA is aborting (this wait or another one timed out).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (uint32_t spin = 1;; ++spin) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((spin & 63u) == 0u) {
-      if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitCycles) {
-        *abort_flag = 1;
-        atomicExch(status, (int)FGR_ERR_DEVICE_TIMEOUT);
-        return false;
-      }
-    }
-  }
-}
-
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
-      : "memory");
-}
-
-__device__ __forceinline__ void tcgen05_alloc(uint32_t dst_smem, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tcgen05_relinquish() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tcgen05_dealloc(uint32_t taddr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tcgen05_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate; `accumulate` = 0 overwrites D.
-__device__ __forceinline__ void tcgen05_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                                 uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// 32 lanes x 16 consecutive 32-bit columns: thread i of the warp gets lane (base + i), register j = column j.
-__device__ __forceinline__ void tcgen05_ld16(uint32_t taddr, float* v) {
-  uint32_t r[16];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
-}
-
-// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes, stored with the
-// 128-byte swizzle (what a TMA load with the 128B swizzle mode leaves in shared memory): groups of
-// 8 rows are 1024 bytes apart (stride byte offset); the leading byte offset is unused for this
-// layout; descriptor version 1; layout type 2 = 128-byte swizzle.
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);   // start address, 16-byte units
-  d |= (uint64_t)1 << 16;                     // leading byte offset (ignored for swizzled K-major)
-  d |= (uint64_t)(1024 >> 4) << 32;           // stride byte offset
-  d |= (uint64_t)1 << 46;                     // version
-  d |= (uint64_t)2 << 61;                     // 128-byte swizzle
-  return d;
-}
-// Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = tile_n.
-__device__ __forceinline__ uint32_t make_idesc(int tile_n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(tile_n >> 3) << 17) | ((uint32_t)(kUmmaTileM >> 4) << 24);
-}
-
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ float activation(int act, float u) {
-  if (act == FGR_ACT_RELU) return fmaxf(u, 0.0f);
-  if (act == FGR_ACT_GELU_TANH) {
-    // 0.5 u (1 + tanh t) = u / (1 + exp(-2 t)),  t = sqrt(2/pi) (u + 0.044715 u^3)
-    const float k = -2.0f * 0.7978845608028654f * 1.4426950408889634f;   // -2 sqrt(2/pi) log2(e)
-    float t = k * (u + 0.044715f * u * u * u);
-    return __fdividef(u, 1.0f + ex2(t));
-  }
-  return u;
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 r = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&r);
-}
-
-struct TileCoord { int bt, m0, n0; };
-__device__ __forceinline__ TileCoord tile_coord(long long t, const Params& p) {
-  TileCoord c;
-  const int per_batch = p.tiles_m * p.tiles_n;
-  c.bt = (int)(t / per_batch);
-  const int r = (int)(t - (long long)c.bt * per_batch);
-  c.m0 = (r / p.tiles_n) * kUmmaTileM;    // N fastest: the tiles of one row block are worked on together
-  c.n0 = (r % p.tiles_n) * p.tile_n;
-  return c;
-}
-
-// ------------------------------------------------------------------------------------------ kernel
-__global__ void __launch_bounds__(kUmmaThreads, 1)
-umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const Params p) {
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-  const UmmaSmem L = umma_smem_layout(p.tile_n, p.stages);
-
-  float* vec_s = reinterpret_cast<float*>(base_ptr + L.vec_off);   // [epilogue warp][bias|scale][128]
-  const uint32_t bar_base = base + L.bar_off;
-  auto full_bar = [&](int s) { return bar_base + 8u * s; };
-  auto empty_bar = [&](int s) { return bar_base + 8u * (kUmmaMaxStages + s); };
-  auto tmem_full_bar = [&](int b) { return bar_base + 8u * (2 * kUmmaMaxStages + b); };
-  auto tmem_empty_bar = [&](int b) { return bar_base + 8u * (2 * kUmmaMaxStages + 2 + b); };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L.misc_off);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L.misc_off + 4);
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int kblocks = (p.K + kUmmaBlockK - 1) / kUmmaBlockK;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tmem_full_bar(b), 1); mbar_init(tmem_empty_bar(b), 8); }
-    *abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
-  if (warp == 1) {
-    tcgen05_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
-    tcgen05_relinquish();
-  }
-  tcgen05_fence_before();
-  __syncthreads();
-  tcgen05_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-
-  if (warp == 0) {
-    // ================================================================ TMA producer
-    if (lane == 0) {
-      uint32_t it = 0;
-      bool ok = true;
-      for (long long t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x) {
-        const TileCoord c = tile_coord(t, p);
-        for (int kb = 0; kb < kblocks; ++kb, ++it) {
-          const int s = it % p.stages;
-          const uint32_t ph = (it / p.stages) & 1u;
-          if (!(ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status))) break;
-          mbar_arrive_expect_tx(full_bar(s), (uint32_t)L.stage_bytes);
-          const uint32_t xs = base + (uint32_t)(s * L.stage_bytes);
-          tma_load_3d(xs, &tmap_x, kb * kUmmaBlockK, c.m0, c.bt, full_bar(s));
-          tma_load_3d(xs + L.x_bytes, &tmap_w, kb * kUmmaBlockK, c.n0, c.bt, full_bar(s));
-        }
-      }
-      if (!ok) {
-        // Aborting: let the copies already issued land before the CTA gives its shared memory back.
-        const uint32_t issued = it < (uint32_t)p.stages ? it : (uint32_t)p.stages;
-        for (uint32_t j = 0; j < issued; ++j) {
-          const uint32_t i2 = it - 1 - j;
-          const long long t0 = clock64();
-          while (!mbar_try_wait(full_bar(i2 % p.stages), (i2 / p.stages) & 1u))
-            if (clock64() - t0 > kWaitCycles / 8) break;
-        }
-      }
-    }
-  } else if (warp == 1) {
-    // ================================================================ MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc = make_idesc(p.tile_n);
-      uint32_t it = 0, tcount = 0;
-      bool ok = true;
-      for (long long t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x, ++tcount) {
-        const uint32_t buf = tcount & 1u, aph = (tcount >> 1) & 1u;
-        if (!(ok = mbar_wait(tmem_empty_bar(buf), aph ^ 1u, abort_flag, p.status))) break;
-        tcgen05_fence_after();
-        const uint32_t d = tmem_base + buf * 256u;
-        for (int kb = 0; kb < kblocks; ++kb, ++it) {
-          const int s = it % p.stages;
-          const uint32_t ph = (it / p.stages) & 1u;
-          if (!(ok = mbar_wait(full_bar(s), ph, abort_flag, p.status))) break;
-          tcgen05_fence_after();
-          const uint32_t xs = base + (uint32_t)(s * L.stage_bytes);
-          const uint64_t a0 = make_smem_desc(xs), b0 = make_smem_desc(xs + L.x_bytes);
-#pragma unroll
-          for (int k = 0; k < kUmmaBlockK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor address units
-            tcgen05_mma_bf16(d, a0 + 2u * k, b0 + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
-          tcgen05_commit(empty_bar(s));
-        }
-        if (ok) tcgen05_commit(tmem_full_bar(buf));
-      }
-    }
-  } else {
-    // ================================================================ epilogue (warps 2..9)
-    const int ew = warp - 2;
-    const int quad = warp & 3;              // TMEM lanes a warp may read: 32 * (warp id % 4) ...
-    const int half = ew >> 2;               // which part of the tile's columns
-    float* bias_s = vec_s + ew * 256;       // this warp's staging: [bias | scale][128]
-    float* scale_s = bias_s + 128;
-    const int c_begin = half ? p.half_n : 0;
-    const int c_end = half ? p.tile_n : p.half_n;
-    const bool exp_kind = p.reduce != FGR_RED_MAXSUM;
-    const bool softmax = p.reduce == FGR_RED_SOFTMAX;
-    const bool store_y = p.write_y && !softmax;
-    const float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
-    uint32_t tcount = 0;
-    bool ok = true;
-    for (long long t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x, ++tcount) {
-      const TileCoord c = tile_coord(t, p);
-      const uint32_t buf = tcount & 1u, aph = (tcount >> 1) & 1u;
-      // stage the bias and scale of this warp's columns in its own slice of shared memory
-      for (int i = lane; i < c_end - c_begin; i += 32) {
-        const int n = c.n0 + c_begin + i;
-        float b = 0.0f, s = 1.0f;
-        if (n < p.N) {
-          if (p.bias) b = p.bias[(p.bias_per_batch ? (long long)c.bt * p.N : 0) + n];
-          if (p.scale_kind == FGR_SCALE_PER_COLUMN) s = p.scale_vec[n];
-          else if (p.scale_kind == FGR_SCALE_SCALAR) s = p.scale;
-        }
-        bias_s[i] = b;
-        scale_s[i] = s;
-      }
-      __syncwarp();
-      ok = __all_sync(0xffffffffu, mbar_wait(tmem_full_bar(buf), aph, abort_flag, p.status));
-      if (!ok) break;
-      tcgen05_fence_after();
-
-      const int m = c.m0 + quad * 32 + lane;
-      const bool row_ok = m < p.M;
-      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * 256u;
-      __nv_bfloat16* yrow = static_cast<__nv_bfloat16*>(p.Y) + (long long)c.bt * p.bsy + (long long)m * p.ldy + c.n0;
-      const int n_valid = p.N - c.n0;       // columns of this tile inside the matrix (may exceed tile_n)
-
-      float r0 = -CUDART_INF_F, r1 = 0.0f;  // (max, sum) or (max in log2 units, sum of 2^(t - max))
-      float v[kChunk];
-      if (softmax) {
-        // pass A: row maximum over this warp's columns
-        for (int cc = c_begin; cc < c_end && cc < n_valid; cc += kChunk) {
-          tcgen05_ld16(taddr + cc, v);
-          const int nv = n_valid - cc;
-#pragma unroll
-          for (int j = 0; j < kChunk; ++j) {
-            float y = activation(p.act, v[j] + bias_s[cc - c_begin + j]) * scale_s[cc - c_begin + j];
-            if (j < nv) r0 = fmaxf(r0, y * kLog2e);
-          }
-        }
-        // pass B: exponentials relative to that maximum, their sum, and the bf16 store
-        for (int cc = c_begin; cc < c_end && cc < n_valid; cc += kChunk) {
-          tcgen05_ld16(taddr + cc, v);
-          const int nv = n_valid - cc;
-          float e[kChunk];
-#pragma unroll
-          for (int j = 0; j < kChunk; ++j) {
-            float y = activation(p.act, v[j] + bias_s[cc - c_begin + j]) * scale_s[cc - c_begin + j];
-            e[j] = (j < nv) ? ex2(y * kLog2e - r0) : 0.0f;
-            r1 += e[j];
-          }
-          if (row_ok) {
-            uint4 q0 = make_uint4(pack_bf16(e[0], e[1]), pack_bf16(e[2], e[3]), pack_bf16(e[4], e[5]), pack_bf16(e[6], e[7]));
-            *reinterpret_cast<uint4*>(yrow + cc) = q0;
-            if (nv > 8) {
-              uint4 q1 = make_uint4(pack_bf16(e[8], e[9]), pack_bf16(e[10], e[11]), pack_bf16(e[12], e[13]), pack_bf16(e[14], e[15]));
-              *reinterpret_cast<uint4*>(yrow + cc + 8) = q1;
-            }
-          }
-        }
-      } else {
-        for (int cc = c_begin; cc < c_end && cc < n_valid; cc += kChunk) {
-          tcgen05_ld16(taddr + cc, v);
-          const int nv = n_valid - cc;
-          float y[kChunk];
-#pragma unroll
-          for (int j = 0; j < kChunk; ++j) y[j] = activation(p.act, v[j] + bias_s[cc - c_begin + j]) * scale_s[cc - c_begin + j];
-          if (store_y && row_ok) {
-            uint4 q0 = make_uint4(pack_bf16(y[0], y[1]), pack_bf16(y[2], y[3]), pack_bf16(y[4], y[5]), pack_bf16(y[6], y[7]));
-            *reinterpret_cast<uint4*>(yrow + cc) = q0;
-            if (nv > 8) {
-              uint4 q1 = make_uint4(pack_bf16(y[8], y[9]), pack_bf16(y[10], y[11]), pack_bf16(y[12], y[13]), pack_bf16(y[14], y[15]));
-              *reinterpret_cast<uint4*>(yrow + cc + 8) = q1;
-            }
-          }
-          if (exp_kind) {
-            float cm = -CUDART_INF_F;
-#pragma unroll
-            for (int j = 0; j < kChunk; ++j) { y[j] *= kLog2e; if (j < nv) cm = fmaxf(cm, y[j]); }
-            const float mn = fmaxf(r0, cm);
-            float l = 0.0f;
-#pragma unroll
-            for (int j = 0; j < kChunk; ++j) l += (j < nv) ? ex2(y[j] - mn) : 0.0f;
-            r1 = r1 * ex2(r0 - mn) + l;
-            r0 = mn;
-          } else {
-#pragma unroll
-            for (int j = 0; j < kChunk; ++j) if (j < nv) { r0 = fmaxf(r0, y[j]); r1 += y[j]; }
-          }
-        }
-      }
-      // accumulator buffer drained: hand it back to the MMA warp
-      tcgen05_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(tmem_empty_bar(buf));
-
-      if (row_ok) {
-        if (exp_kind) r0 *= kLn2;           // back to natural-log units; r1 is unchanged by the change of base
-        const int tn = c.n0 / p.tile_n;
-        float2* dst = reinterpret_cast<float2*>(p.parts) + ((long long)c.bt * p.M + m) * p.parts_per_row + tn * 2 + half;
-        *dst = make_float2(r0, r1);
-      }
-    }
-  }
-
-  tcgen05_fence_before();
-  __syncthreads();
-  if (warp == 1) tcgen05_dealloc(tmem_base, kTmemCols);
-}
-
-}  // namespace
 
 cudaError_t umma_prepare(int) {
-  return cudaFuncSetAttribute(umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+  cudaError_t e = umma_prepare_act_none();
+  if (e == cudaSuccess) e = umma_prepare_act_relu();
+  if (e == cudaSuccess) e = umma_prepare_act_gelu();
+  return e;
 }
 
 cudaError_t launch_umma(const Params& p, const void* tmap_x, const void* tmap_w, int grid, int smem_bytes,
                         cudaStream_t stream) {
-  umma_kernel<<<grid, kUmmaThreads, smem_bytes, stream>>>(*static_cast<const CUtensorMap*>(tmap_x),
-                                                          *static_cast<const CUtensorMap*>(tmap_w), p);
-  return cudaGetLastError();
+  const bool softmax = p.reduce == FGR_RED_SOFTMAX;
+  const bool exp_kind = p.reduce != FGR_RED_MAXSUM;
+  const bool wy = p.write_y && !softmax;
+  // exp kinds that do not store y fold log2(e) into the staged scale vector, so they always multiply
+  const bool sc = (exp_kind && !wy) || p.scale_kind != FGR_SCALE_NONE;
+  switch (p.act) {
+    case FGR_ACT_NONE: return umma_launch_act_none(sc, p.reduce, wy, p, tmap_x, tmap_w, grid, smem_bytes, stream);
+    case FGR_ACT_RELU: return umma_launch_act_relu(sc, p.reduce, wy, p, tmap_x, tmap_w, grid, smem_bytes, stream);
+    case FGR_ACT_GELU_TANH: return umma_launch_act_gelu(sc, p.reduce, wy, p, tmap_x, tmap_w, grid, smem_bytes, stream);
+    default: return cudaErrorInvalidValue;
+  }
 }
 
 }  // namespace fgr
