@@ -89,17 +89,20 @@ typedef struct fgr_desc {
   int32_t device;          /* CUDA device ordinal */
   int32_t force_path;      /* fgr_path; FGR_PATH_AUTO lets the shape decide */
   int32_t force_tile_n;    /* 0 = automatic; else the N extent of a tcgen05 tile (multiple of 16, 16..256) */
+  int32_t force_cta_pair;  /* 0 = automatic; 1 = every CTA alone (128-row tiles); 2 = clusters of two CTAs
+                              sharing 256-row tiles (tcgen05 cta_group::2; needs tile_n % 32 == 0) */
 } fgr_desc;
 
 /* What fgr_plan / fgr_create decided; plain host data, for callers, tests and benchmarks. */
 typedef struct fgr_plan_info {
   int32_t path;            /* fgr_path actually used */
-  int32_t tile_m, tile_n;  /* output tile of one CTA */
+  int32_t tile_m, tile_n;  /* output tile of one CTA, or of one CTA pair (tile_m = 256) */
   int32_t stages;          /* depth of the shared-memory operand ring (0 for SIMT paths) */
   int32_t parts_per_row;   /* number of split-N partial pairs per row in the workspace */
   int32_t grid;            /* CTAs of the main kernel */
   int32_t launches;        /* kernels launched by one fgr_run */
   int32_t smem_bytes;      /* dynamic shared memory of the main kernel */
+  int32_t cta_pair;        /* 2 if the main kernel runs as clusters of two CTAs, else 1 */
   int64_t num_tiles;       /* output tiles in the problem */
   uint64_t workspace_bytes;/* what fgr_run needs */
   double flop;             /* 2 * batch * M * N * K */

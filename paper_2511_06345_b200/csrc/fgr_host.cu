@@ -82,6 +82,7 @@ int validate(const fgr_desc* d) {
                        r.bsy < (long long)(d->M - 1) * r.ldy + d->N))
     return FGR_ERR_INVALID_ARG;
   if ((long long)d->batch * d->M > (1LL << 31) - 1) return FGR_ERR_UNSUPPORTED;
+  if (d->force_cta_pair < 0 || d->force_cta_pair > 2) return FGR_ERR_INVALID_ARG;
   if (d->force_tile_n && (d->force_tile_n % 16 || d->force_tile_n < 16 || d->force_tile_n > 256)) return FGR_ERR_INVALID_ARG;
   return FGR_OK;
 }
@@ -146,21 +147,30 @@ int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
     pi.smem_bytes = 0;
     if (p.tiles_m > 65535 || d.batch > 65535) return FGR_ERR_UNSUPPORTED;
   } else {
-    p.tiles_m = (d.M + kUmmaTileM - 1) / kUmmaTileM;
     int tn = d.force_tile_n;
+    const int row_blocks = (d.M + kUmmaTileM - 1) / kUmmaTileM;
     if (!tn) {
-      if (path == FGR_PATH_UMMA_STREAM_W) tn = pick_stream_tile_n((long long)d.batch * p.tiles_m, d.N, sms);
+      if (path == FGR_PATH_UMMA_STREAM_W) tn = pick_stream_tile_n((long long)d.batch * row_blocks, d.N, sms);
       else tn = d.N >= 256 ? 256 : ((d.N + 15) / 16) * 16;
     }
+    // CTA pairs (256-row tiles, one tcgen05.mma.cta_group::2 for two SMs) cut the operand traffic
+    // per SM by a third; they need at least two row blocks and a W tile that halves into whole
+    // 16-row groups.
+    int pair = d.force_cta_pair;
+    if (!pair) pair = (path == FGR_PATH_UMMA_TILED && row_blocks >= 2 && tn % 32 == 0 && sms >= 2) ? 2 : 1;
+    if (pair == 2 && tn % 32 != 0) return FGR_ERR_UNSUPPORTED;
+    p.cta_pair = pair;
+    p.tiles_m = (d.M + kUmmaTileM * pair - 1) / (kUmmaTileM * pair);
     p.tile_n = tn;
     p.half_n = ((tn / 2 + 15) / 16) * 16;
     p.slots_per_tile = 2;
     p.tiles_n = (d.N + tn - 1) / tn;
+    const int w_rows = tn / pair;
     int stages = kUmmaMaxStages;
-    while (stages > 1 && umma_smem_layout(tn, stages).total > kSmemLimit) --stages;
+    while (stages > 1 && umma_smem_layout(w_rows, stages).total > kSmemLimit) --stages;
     p.stages = stages;
-    pi.tile_m = kUmmaTileM;
-    pi.smem_bytes = umma_smem_layout(tn, stages).total;
+    pi.tile_m = kUmmaTileM * pair;
+    pi.smem_bytes = umma_smem_layout(w_rows, stages).total;
   }
   p.num_tiles = (long long)d.batch * p.tiles_m * p.tiles_n;
   p.parts_per_row = p.tiles_n * p.slots_per_tile;
@@ -171,8 +181,13 @@ int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
   pi.stages = p.stages;
   pi.parts_per_row = p.parts_per_row;
   pi.num_tiles = p.num_tiles;
-  pi.grid = path == FGR_PATH_SIMT ? (int)(p.num_tiles > 0x7fffffff ? 0x7fffffff : p.num_tiles)
-                                  : (int)(p.num_tiles < sms ? p.num_tiles : sms);
+  if (path == FGR_PATH_SIMT) {
+    pi.grid = (int)(p.num_tiles > 0x7fffffff ? 0x7fffffff : p.num_tiles);
+  } else {
+    const long long groups = sms / p.cta_pair;   // CTAs, or clusters of two
+    pi.grid = (int)(p.num_tiles < groups ? p.num_tiles : groups) * p.cta_pair;
+  }
+  pi.cta_pair = path == FGR_PATH_SIMT ? 1 : p.cta_pair;
   pi.launches = 2;   // main kernel + (merge | softmax normalise)
   pi.workspace_bytes = (uint64_t)kStatusBytes + (uint64_t)d.batch * d.M * p.parts_per_row * 8ull;
   *info = pi;
@@ -316,7 +331,7 @@ int fgr_run(fgr_handle* h, const void* X, const void* W, const float* bias, cons
         h->cached_x = rc == FGR_OK ? X : nullptr;
       }
       if (rc == FGR_OK && W != h->cached_w) {
-        rc = encode_operand(&h->tmap_w, W, d.K, d.N, d.batch, p.ldw, p.bsw, p.tile_n);
+        rc = encode_operand(&h->tmap_w, W, d.K, d.N, d.batch, p.ldw, p.bsw, p.tile_n / p.cta_pair);
         h->cached_w = rc == FGR_OK ? W : nullptr;
       }
       if (rc == FGR_OK) e = launch_umma(p, &h->tmap_x, &h->tmap_w, h->plan.grid, h->plan.smem_bytes, stream);

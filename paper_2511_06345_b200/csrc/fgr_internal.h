@@ -37,6 +37,7 @@ struct Params {
   int tiles_m, tiles_n;
   long long num_tiles;
   int stages;
+  int cta_pair;        // tcgen05 paths: 1 = each CTA works alone, 2 = clusters of two CTAs share 256-row tiles
 };
 
 // Column -> partial-slot mapping shared by the producers of the partials and the normalise pass.
@@ -54,10 +55,11 @@ struct UmmaSmem {
   int misc_off;     // TMEM base address, abort flag
   int total;        // bytes to request (includes 1024 of alignment slack)
 };
-__host__ __device__ inline UmmaSmem umma_smem_layout(int tile_n, int stages) {
+// `w_rows`: rows of the W tile one CTA loads per k-block (tile_n, or tile_n / 2 for a CTA pair).
+__host__ __device__ inline UmmaSmem umma_smem_layout(int w_rows, int stages) {
   UmmaSmem s;
   s.x_bytes = kUmmaTileM * kUmmaBlockK * 2;
-  s.w_bytes = tile_n * kUmmaBlockK * 2;
+  s.w_bytes = w_rows * kUmmaBlockK * 2;
   s.stage_bytes = s.x_bytes + s.w_bytes;
   s.vec_off = s.stage_bytes * stages;
   s.bar_off = s.vec_off + 8 * 2 * 128 * 4;

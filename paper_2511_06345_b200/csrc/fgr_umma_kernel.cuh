@@ -117,6 +117,57 @@ __device__ __forceinline__ void tcgen05_ld16_issue(uint32_t taddr, uint32_t* r) 
       : "memory");
 }
 __device__ __forceinline__ void tcgen05_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// ---- CTA pairs (cluster of two CTAs driving one tcgen05.mma.cta_group::2).  Within a cluster of
+// two, a shared-memory address of the odd CTA differs from the same offset in the even CTA by
+// bit 24; clearing it names the even (leader) CTA's copy.
+constexpr uint32_t kPeerBitMask = 0xFEFFFFFFu;
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  __syncwarp();
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA load whose completion bytes are counted on the LEADER CTA's mbarrier (same offset as `bar`).
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar & kPeerBitMask)
+      : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_leader(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar & kPeerBitMask) : "memory");
+}
+__device__ __forceinline__ void tcgen05_alloc_pair(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tcgen05_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tcgen05_dealloc_pair(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// Arrives (once all MMAs issued so far have completed) on the barrier at this offset in BOTH CTAs.
+__device__ __forceinline__ void tcgen05_commit_pair(uint32_t bar) {
+  asm volatile(
+      "{\n\t.reg .b16 m;\n\tmov.b16 m, 3;\n\t"
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], m;\n\t}"
+      ::"r"(bar)
+      : "memory");
+}
+// D (256 rows: 128 in each CTA's tensor memory) (+)= A (128 rows from each CTA) * B^T (tile_n / 2 rows from each CTA)
+__device__ __forceinline__ void tcgen05_mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                      uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
@@ -134,9 +185,10 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
   d |= (uint64_t)2 << 61;                     // 128-byte swizzle
   return d;
 }
-// Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = tile_n.
-__device__ __forceinline__ uint32_t make_idesc(int tile_n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(tile_n >> 3) << 17) | ((uint32_t)(kUmmaTileM >> 4) << 24);
+// Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = 128 (256 for a CTA
+// pair), N = tile_n.
+__device__ __forceinline__ uint32_t make_idesc(int tile_m, int tile_n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(tile_n >> 3) << 17) | ((uint32_t)(tile_m >> 4) << 24);
 }
 
 __device__ __forceinline__ float ex2(float x) {
@@ -171,13 +223,15 @@ __device__ __forceinline__ void store_bf16x16(__nv_bfloat16* dst, const float* y
         make_uint4(pack_bf16(y[8], y[9]), pack_bf16(y[10], y[11]), pack_bf16(y[12], y[13]), pack_bf16(y[14], y[15]));
 }
 
+// Work unit t -> (batch, first row of this CTA, first column).  A unit is one 128-row tile, or for
+// a CTA pair a 256-row tile of which CTA `rank` owns rows [128 rank, 128 rank + 128).
 struct TileCoord { int bt, m0, n0; };
-__device__ __forceinline__ TileCoord tile_coord(long long t, const Params& p) {
+__device__ __forceinline__ TileCoord tile_coord(long long t, const Params& p, int rank) {
   TileCoord c;
   const int per_batch = p.tiles_m * p.tiles_n;
   c.bt = (int)(t / per_batch);
   const int r = (int)(t - (long long)c.bt * per_batch);
-  c.m0 = (r / p.tiles_n) * kUmmaTileM;    // N fastest: the tiles of one row block are worked on together
+  c.m0 = (r / p.tiles_n) * (kUmmaTileM * p.cta_pair) + rank * kUmmaTileM;   // N fastest
   c.n0 = (r % p.tiles_n) * p.tile_n;
   return c;
 }
@@ -216,14 +270,24 @@ __device__ __forceinline__ void apply16(const uint32_t* r, const float* bias_s, 
 }
 
 // ------------------------------------------------------------------------------------------ kernel
-template <int ACT, bool SC, int RED, bool WY>
+// PAIR = false: every CTA works alone on 128 x tile_n tiles (tcgen05 cta_group::1).
+// PAIR = true : the grid is launched in clusters of two CTAs that share 256 x tile_n tiles.  Each
+//   CTA loads its own 128 rows of X and half (tile_n / 2 rows) of the W tile; the even CTA (the
+//   leader) issues tcgen05.mma.cta_group::2, which reads both CTAs' shared memory and writes rows
+//   [0, 128) of the tile to its own tensor memory and rows [128, 256) to its peer's.  Per CTA and
+//   k-block that is 32 KB of operands instead of 48 KB for the same tensor work.  Barriers:
+//   "full" lives in the leader (both CTAs' TMA loads count their bytes there), "empty" and
+//   "tmem_full" are signalled in both CTAs by one multicast tcgen05.commit, "tmem_empty" lives in
+//   the leader and collects the epilogue warps of both CTAs.
+template <int ACT, bool SC, int RED, bool WY, bool PAIR>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const Params p) {
   using V = Variant<ACT, SC, RED, WY>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-  const UmmaSmem L = umma_smem_layout(p.tile_n, p.stages);
+  const int w_rows = PAIR ? p.tile_n / 2 : p.tile_n;       // rows of the W tile this CTA loads
+  const UmmaSmem L = umma_smem_layout(w_rows, p.stages);
 
   float* vec_s = reinterpret_cast<float*>(base_ptr + L.vec_off);   // [epilogue warp][bias|scale][128]
   const uint32_t bar_base = base + L.bar_off;
@@ -236,22 +300,32 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kblocks = (p.K + kUmmaBlockK - 1) / kUmmaBlockK;
+  const int rank = PAIR ? (int)cluster_ctarank() : 0;      // 0 = leader
+  // work units are dealt round-robin to CTAs (PAIR: to clusters)
+  const long long unit0 = PAIR ? (long long)(blockIdx.x >> 1) : (long long)blockIdx.x;
+  const long long unit_step = PAIR ? (long long)(gridDim.x >> 1) : (long long)gridDim.x;
 
   if (threadIdx.x == 0) {
     prefetch_tensormap(&tmap_x);
     prefetch_tensormap(&tmap_w);
     for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tmem_full_bar(b), 1); mbar_init(tmem_empty_bar(b), 8); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tmem_full_bar(b), 1); mbar_init(tmem_empty_bar(b), PAIR ? 16 : 8); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    tcgen05_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
-    tcgen05_relinquish();
+    if constexpr (PAIR) {
+      tcgen05_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+      tcgen05_relinquish_pair();
+    } else {
+      tcgen05_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+      tcgen05_relinquish();
+    }
   }
   tcgen05_fence_before();
   __syncthreads();
+  if constexpr (PAIR) cluster_sync_all();   // the peer's barriers exist before anything signals them
   tcgen05_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -260,20 +334,28 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (long long t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x) {
-        const TileCoord c = tile_coord(t, p);
+      for (long long t = unit0; t < p.num_tiles && ok; t += unit_step) {
+        const TileCoord c = tile_coord(t, p, rank);
         for (int kb = 0; kb < kblocks; ++kb, ++it) {
           const int s = it % p.stages;
           const uint32_t ph = (it / p.stages) & 1u;
           if (!(ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status))) break;
-          mbar_arrive_expect_tx(full_bar(s), (uint32_t)L.stage_bytes);
           const uint32_t xs = base + (uint32_t)(s * L.stage_bytes);
-          tma_load_3d(xs, &tmap_x, kb * kUmmaBlockK, c.m0, c.bt, full_bar(s));
-          tma_load_3d(xs + L.x_bytes, &tmap_w, kb * kUmmaBlockK, c.n0, c.bt, full_bar(s));
+          if constexpr (PAIR) {
+            if (rank == 0) mbar_arrive_expect_tx(full_bar(s), 2u * (uint32_t)L.stage_bytes);
+            tma_load_3d_pair(xs, &tmap_x, kb * kUmmaBlockK, c.m0, c.bt, full_bar(s));
+            tma_load_3d_pair(xs + L.x_bytes, &tmap_w, kb * kUmmaBlockK, c.n0 + rank * w_rows, c.bt, full_bar(s));
+          } else {
+            mbar_arrive_expect_tx(full_bar(s), (uint32_t)L.stage_bytes);
+            tma_load_3d(xs, &tmap_x, kb * kUmmaBlockK, c.m0, c.bt, full_bar(s));
+            tma_load_3d(xs + L.x_bytes, &tmap_w, kb * kUmmaBlockK, c.n0, c.bt, full_bar(s));
+          }
         }
       }
-      if (!ok) {
+      if (!ok && !PAIR) {
         // Aborting: let the copies already issued land before the CTA gives its shared memory back.
+        // (A pair ends with a cluster-wide barrier and its copies are counted in the leader, so
+        // there the wait for the peer serves the same purpose.)
         const uint32_t issued = it < (uint32_t)p.stages ? it : (uint32_t)p.stages;
         for (uint32_t j = 0; j < issued; ++j) {
           const uint32_t i2 = it - 1 - j;
@@ -284,12 +366,12 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
       }
     }
   } else if (warp == 1) {
-    // ================================================================ MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc = make_idesc(p.tile_n);
+    // ================================================================ MMA issuer (the leader CTA of a pair)
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc = make_idesc(PAIR ? 2 * kUmmaTileM : kUmmaTileM, p.tile_n);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (long long t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x, ++tcount) {
+      for (long long t = unit0; t < p.num_tiles && ok; t += unit_step, ++tcount) {
         const uint32_t buf = tcount & 1u, aph = (tcount >> 1) & 1u;
         if (!(ok = mbar_wait(tmem_empty_bar(buf), aph ^ 1u, abort_flag, p.status))) break;
         tcgen05_fence_after();
@@ -302,11 +384,15 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
           const uint32_t xs = base + (uint32_t)(s * L.stage_bytes);
           const uint64_t a0 = make_smem_desc(xs), b0 = make_smem_desc(xs + L.x_bytes);
 #pragma unroll
-          for (int k = 0; k < kUmmaBlockK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor address units
-            tcgen05_mma_bf16(d, a0 + 2u * k, b0 + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
-          tcgen05_commit(empty_bar(s));
+          for (int k = 0; k < kUmmaBlockK / 16; ++k) {   // 16 bf16 = 32 bytes = 2 descriptor address units
+            if constexpr (PAIR) tcgen05_mma_bf16_pair(d, a0 + 2u * k, b0 + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            else tcgen05_mma_bf16(d, a0 + 2u * k, b0 + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          if constexpr (PAIR) tcgen05_commit_pair(empty_bar(s)); else tcgen05_commit(empty_bar(s));
         }
-        if (ok) tcgen05_commit(tmem_full_bar(buf));
+        if (ok) {
+          if constexpr (PAIR) tcgen05_commit_pair(tmem_full_bar(buf)); else tcgen05_commit(tmem_full_bar(buf));
+        }
       }
     }
   } else {
@@ -320,8 +406,8 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
     const int c_end = half ? p.tile_n : p.half_n;
     uint32_t tcount = 0;
     bool ok = true;
-    for (long long t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x, ++tcount) {
-      const TileCoord c = tile_coord(t, p);
+    for (long long t = unit0; t < p.num_tiles && ok; t += unit_step, ++tcount) {
+      const TileCoord c = tile_coord(t, p, rank);
       const uint32_t buf = tcount & 1u, aph = (tcount >> 1) & 1u;
       // stage the bias and scale of this warp's columns in its own slice of shared memory
       for (int i = lane; i < c_end - c_begin; i += 32) {
@@ -413,7 +499,9 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
       // accumulator buffer drained: hand it back to the MMA warp
       tcgen05_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tmem_empty_bar(buf));
+      if (lane == 0) {
+        if constexpr (PAIR) mbar_arrive_leader(tmem_empty_bar(buf)); else mbar_arrive(tmem_empty_bar(buf));
+      }
 
       if (row_ok) {
         if constexpr (V::kExp) r0 *= kLn2;   // back to natural-log units; r1 is unchanged by the change of base
@@ -426,18 +514,42 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
 
   tcgen05_fence_before();
   __syncthreads();
-  if (warp == 1) tcgen05_dealloc(tmem_base, kTmemCols);
+  if constexpr (PAIR) {
+    // neither CTA may leave while its peer can still read its shared memory or signal its barriers
+    cluster_sync_all();
+    if (warp == 1) tcgen05_dealloc_pair(tmem_base, kTmemCols);
+  } else {
+    if (warp == 1) tcgen05_dealloc(tmem_base, kTmemCols);
+  }
 }
 
 // ------------------------------------------------------------------------------------------ host
 template <int ACT, bool SC, int RED, bool WY>
 cudaError_t launch_one(const Params& p, const CUtensorMap& tx, const CUtensorMap& tw, int grid, int smem, cudaStream_t s) {
-  umma_kernel<ACT, SC, RED, WY><<<grid, kUmmaThreads, smem, s>>>(tx, tw, p);
+  if (p.cta_pair == 2) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kUmmaThreads);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, umma_kernel<ACT, SC, RED, WY, true>, tx, tw, p);
+  }
+  umma_kernel<ACT, SC, RED, WY, false><<<grid, kUmmaThreads, smem, s>>>(tx, tw, p);
   return cudaGetLastError();
 }
 template <int ACT, bool SC, int RED, bool WY>
 cudaError_t prepare_one() {
-  return cudaFuncSetAttribute(umma_kernel<ACT, SC, RED, WY>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+  cudaError_t e = cudaFuncSetAttribute(umma_kernel<ACT, SC, RED, WY, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(umma_kernel<ACT, SC, RED, WY, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+  return e;
 }
 
 // The variants that exist per activation.  Exp kinds that do not store y always multiply by the

@@ -34,8 +34,8 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_struct_layout_matches_header():
-    assert ctypes.sizeof(fgr.fgr_desc) == 112      # the value sizeof(fgr_desc) has in C (gcc, x86-64)
-    assert ctypes.sizeof(fgr.fgr_plan_info) == 64
+    assert ctypes.sizeof(fgr.fgr_desc) == 120      # the value sizeof(fgr_desc) has in C (gcc, x86-64)
+    assert ctypes.sizeof(fgr.fgr_plan_info) == 72
     assert fgr.fgr_status_string(0) == "ok" and "wait" in fgr.fgr_status_string(fgr.FGR_ERR_DEVICE_TIMEOUT)
     assert fgr.fgr_path_name(fgr.FGR_PATH_UMMA_STREAM_W) == "umma_stream_w"
 
@@ -48,18 +48,18 @@ def test_path_selection_for_the_five_workloads():
     c1 = _plan(1, 256, 256, 256, fgr.FGR_F32, fgr.FGR_ACT_GELU_TANH, 0, fgr.FGR_RED_LSE)
     assert c1.path == fgr.FGR_PATH_SIMT and c1.parts_per_row == 4 and c1.num_tiles == 16
     c2 = _plan(1, 4096, 4096, 4096, fgr.FGR_BF16, fgr.FGR_ACT_RELU, 2, fgr.FGR_RED_MAXSUM, write_y=1)
-    assert c2.path == fgr.FGR_PATH_UMMA_TILED and (c2.tile_m, c2.tile_n) == (128, 256)
-    assert c2.num_tiles == 512 and c2.grid == 148 and c2.parts_per_row == 32
+    assert c2.path == fgr.FGR_PATH_UMMA_TILED and (c2.tile_m, c2.tile_n) == (256, 256) and c2.cta_pair == 2
+    assert c2.num_tiles == 256 and c2.grid == 148 and c2.parts_per_row == 32 and c2.stages == 6
     assert c2.workspace_bytes == 256 + 4096 * 32 * 8 and c2.flop == 2.0 * 4096 ** 3
     assert c2.min_bytes == 3 * 4096 * 4096 * 2 + 2 * 4096 * 4 + 4096 * 2 * 4
     c3 = _plan(1, 8192, 8192, 2048, fgr.FGR_BF16, 0, 1, fgr.FGR_RED_SOFTMAX, scale=2048 ** -0.5)
     assert c3.path == fgr.FGR_PATH_UMMA_TILED and c3.parts_per_row == 64
     c4 = _plan(1, 128, 16384, 8192, fgr.FGR_BF16, 2, 0, fgr.FGR_RED_LSE)
-    assert c4.path == fgr.FGR_PATH_UMMA_STREAM_W
+    assert c4.path == fgr.FGR_PATH_UMMA_STREAM_W and c4.cta_pair == 1
     assert c4.num_tiles <= 148 and c4.num_tiles >= 140          # one wave that fills the machine
     assert c4.stages >= 6 and c4.smem_bytes <= 232448
     c5 = _plan(32, 1024, 1024, 512, fgr.FGR_BF16, 1, 0, fgr.FGR_RED_MAXSUM)
-    assert c5.path == fgr.FGR_PATH_UMMA_TILED and c5.num_tiles == 1024
+    assert c5.path == fgr.FGR_PATH_UMMA_TILED and c5.num_tiles == 512 and c5.cta_pair == 2
     small_sm = fgr.fgr_plan(fgr.make_desc(1, 128, 16384, 8192, fgr.FGR_BF16, 2, 0, 0), 64)
     assert small_sm.grid <= 64
 
@@ -67,6 +67,13 @@ def test_path_selection_for_the_five_workloads():
 def test_forced_tiles_and_paths():
     p = _plan(1, 300, 520, 200, fgr.FGR_BF16, 0, 0, 0, force_path=fgr.FGR_PATH_UMMA_TILED, force_tile_n=112)
     assert p.tile_n == 112 and p.parts_per_row == 2 * 5 and p.num_tiles == 3 * 5
+    p = _plan(1, 300, 520, 200, fgr.FGR_BF16, 0, 0, 0, force_path=fgr.FGR_PATH_UMMA_TILED, force_cta_pair=1)
+    assert p.cta_pair == 1 and p.tile_m == 128 and p.num_tiles == 3 * 3 and p.stages == 4
+    p = _plan(1, 300, 520, 200, fgr.FGR_BF16, 0, 0, 0, force_path=fgr.FGR_PATH_UMMA_TILED, force_cta_pair=2, force_tile_n=64)
+    assert p.cta_pair == 2 and p.tile_m == 256 and p.num_tiles == 2 * 9 and p.grid == 36
+    with pytest.raises(fgr.FgrError):
+        _plan(1, 300, 520, 200, fgr.FGR_BF16, 0, 0, 0, force_cta_pair=2, force_tile_n=112)   # halves must be whole 16-row groups
+    assert _plan(1, 100, 520, 200, fgr.FGR_BF16, 0, 0, 0, force_path=fgr.FGR_PATH_UMMA_TILED).cta_pair == 1   # one row block
     p = _plan(1, 300, 520, 200, fgr.FGR_BF16, 0, 0, 0, force_path=fgr.FGR_PATH_SIMT)
     assert p.path == fgr.FGR_PATH_SIMT and p.tile_n == 64 and p.parts_per_row == 9
     with pytest.raises(fgr.FgrError) as e:
@@ -84,6 +91,7 @@ def test_forced_tiles_and_paths():
     (dict(ldx=8), fgr.FGR_ERR_INVALID_ARG),           # smaller than K
     (dict(ldy=68), fgr.FGR_ERR_UNSUPPORTED),          # not 16-byte aligned rows
     (dict(force_tile_n=24), fgr.FGR_ERR_INVALID_ARG),
+    (dict(force_cta_pair=3), fgr.FGR_ERR_INVALID_ARG),
     (dict(scale_kind=1, scale=float("inf")), fgr.FGR_ERR_INVALID_ARG),
     (dict(batch=2, bsx=16), fgr.FGR_ERR_INVALID_ARG),  # batches would overlap
 ])

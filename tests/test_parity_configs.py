@@ -30,7 +30,7 @@ def test_c1_full(cuda_device):
 def test_c2_sampled_rows(cuda_device, reduce):
     p = gi.make_config("c2", reduce=reduce)
     Y, out, plan = run_gpu(p)
-    assert plan["path"] == fgr.FGR_PATH_UMMA_TILED and plan["tile_n"] == 256 and plan["grid"] > 100
+    assert plan["path"] == fgr.FGR_PATH_UMMA_TILED and plan["tile_n"] == 256 and plan["grid"] > 100 and plan["cta_pair"] == 2
     rows = _rows(p.M, 128, 40, 2)
     w = compare(p, Y, out, rows=rows)
     assert w["Y"] <= 2e-2 and w["out"] <= 2e-2
@@ -77,7 +77,7 @@ def test_c4_full(cuda_device):
 def test_c5_batched_sampled_rows(cuda_device, reduce):
     p = gi.make_config("c5", reduce=reduce)
     Y, out, plan = run_gpu(p)
-    assert Y is None and plan["num_tiles"] == 1024
+    assert Y is None and plan["num_tiles"] == 512 and plan["cta_pair"] == 2
     rows = _rows(p.batch * p.M, 1024, 48, 6)
     compare(p, Y, out, rows=rows)
     if reduce == gi.RED_MAXSUM:

@@ -74,9 +74,40 @@ def test_umma_tiled(cuda_device, shape, red):
     B, M, N, K, tn = shape
     for i, act in enumerate(ACTS):
         p = _problem(gi.DTYPE_BF16, B, M, N, K, act, (i + red) % 3, red, seed=30 + i, bias_per_batch=i % 2)
-        Y, out, plan = run_gpu(p, force_path=fgr.FGR_PATH_UMMA_TILED, force_tile_n=tn)
-        assert plan["path"] == fgr.FGR_PATH_UMMA_TILED
+        Y, out, plan = run_gpu(p, force_path=fgr.FGR_PATH_UMMA_TILED, force_tile_n=tn, force_cta_pair=1)
+        assert plan["path"] == fgr.FGR_PATH_UMMA_TILED and plan["cta_pair"] == 1
         compare(p, Y, out)
+
+
+PAIR_SHAPES = [
+    # B, M, N, K, force_tile_n: clusters of two CTAs on 256-row tiles (tcgen05 cta_group::2)
+    (1, 256, 256, 64, 0),
+    (1, 129, 264, 72, 0),      # the second CTA of the pair owns a single real row
+    (1, 300, 520, 200, 64),
+    (2, 515, 1000, 136, 96),
+    (1, 1024, 4096, 320, 0),   # more tiles than clusters: persistent loop, both accumulator buffers, ring wrap-around
+]
+
+
+@pytest.mark.parametrize("shape", PAIR_SHAPES)
+@pytest.mark.parametrize("red", REDS)
+def test_umma_cta_pairs(cuda_device, shape, red):
+    B, M, N, K, tn = shape
+    for i, act in enumerate(ACTS):
+        p = _problem(gi.DTYPE_BF16, B, M, N, K, act, (i + red + 1) % 3, red, seed=50 + i, bias_per_batch=(i + 1) % 2)
+        Y, out, plan = run_gpu(p, force_path=fgr.FGR_PATH_UMMA_TILED, force_tile_n=tn, force_cta_pair=2)
+        assert plan["cta_pair"] == 2 and plan["tile_m"] == 256 and plan["grid"] % 2 == 0
+        compare(p, Y, out)
+
+
+def test_cta_pair_and_single_agree_bitwise(cuda_device):
+    """Same tile width, same accumulation order per element: a pair must reproduce single CTAs exactly."""
+    p = _problem(gi.DTYPE_BF16, 1, 700, 1544, 264, gi.ACT_GELU_TANH, gi.SCALE_PER_COLUMN, gi.RED_LSE, seed=55)
+    t = to_device(p)
+    Y1, o1, p1 = run_gpu(p, tensors=t, force_path=fgr.FGR_PATH_UMMA_TILED, force_cta_pair=1)
+    Y2, o2, p2 = run_gpu(p, tensors=t, force_path=fgr.FGR_PATH_UMMA_TILED, force_cta_pair=2)
+    assert p1["cta_pair"] == 1 and p2["cta_pair"] == 2
+    assert np.array_equal(Y1, Y2) and np.array_equal(o1, o2)
 
 
 @pytest.mark.parametrize("red", [gi.RED_LSE, gi.RED_MAXSUM])
