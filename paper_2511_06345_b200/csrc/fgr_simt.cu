@@ -153,17 +153,25 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(const Params p) {
   }
 }
 
-// One warp per row: lane t takes partials t, t + 32, ... in ascending order, then a fixed
-// xor-shuffle tree combines the 32 lanes.  The order never depends on timing: bit-identical
-// results from run to run.
+// Programmatic dependent launch: the kernels below may be made resident while the kernel before
+// them in the stream is still running; this wait returns once that kernel has completed and its
+// writes are visible.  (A no-op for a kernel launched the ordinary way.)
+__device__ __forceinline__ void wait_for_prior_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// G lanes per row (32 / G rows per warp): lane t of a group takes partials t, t + G, ... in ascending
+// order, then a fixed xor-shuffle tree combines the G lanes.  The order never depends on timing:
+// bit-identical results from run to run.
+template <int G>
 __global__ void __launch_bounds__(256) merge_kernel(const Params p) {
-  const long long row = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const int lane = threadIdx.x & 31;
-  if (row >= (long long)p.batch * p.M) return;
-  const float2* src = reinterpret_cast<const float2*>(p.parts) + row * p.parts_per_row;
+  wait_for_prior_kernel();
+  const int lane = threadIdx.x & 31, sub = lane % G;
+  const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const long long row = warp * (32 / G) + lane / G;
+  const bool row_ok = row < (long long)p.batch * p.M;
+  const float2* src = reinterpret_cast<const float2*>(p.parts) + (row_ok ? row : 0) * p.parts_per_row;
   const bool exp_kind = p.reduce != FGR_RED_MAXSUM;
   float a = -CUDART_INF_F, b = 0.0f;
-  for (int t = lane; t < p.parts_per_row; t += 32) {
+  for (int t = sub; t < p.parts_per_row; t += G) {
     float2 v = src[t];
     if (exp_kind) {
       float mn = fmaxf(a, v.x);
@@ -175,7 +183,7 @@ __global__ void __launch_bounds__(256) merge_kernel(const Params p) {
     }
   }
 #pragma unroll
-  for (int o = 16; o >= 1; o >>= 1) {
+  for (int o = G / 2; o >= 1; o >>= 1) {
     float oa = __shfl_xor_sync(0xffffffffu, a, o), ob = __shfl_xor_sync(0xffffffffu, b, o);
     if (exp_kind) {
       float mn = fmaxf(a, oa);
@@ -190,7 +198,7 @@ __global__ void __launch_bounds__(256) merge_kernel(const Params p) {
       b = lo_b + hi_b;
     }
   }
-  if (lane == 0) {
+  if (sub == 0 && row_ok) {
     if (p.reduce == FGR_RED_LSE) p.out[row] = a + logf(b);
     else if (p.reduce != FGR_RED_SOFTMAX) reinterpret_cast<float2*>(p.out)[row] = make_float2(a, b);
   }
@@ -203,6 +211,7 @@ __global__ void __launch_bounds__(256) merge_kernel(const Params p) {
 template <typename T>
 __global__ void __launch_bounds__(256) normalise_kernel(const Params p) {
   extern __shared__ float factor[];   // [parts_per_row]
+  wait_for_prior_kernel();
   const long long row = blockIdx.x;
   const int bt = (int)(row / p.M), m = (int)(row % p.M);
   const float2* src = reinterpret_cast<const float2*>(p.parts) + row * p.parts_per_row;
@@ -271,18 +280,37 @@ cudaError_t launch_simt(const Params& p, cudaStream_t stream) {
   return cudaGetLastError();
 }
 
+// Launch with programmatic stream serialization: the kernel may become resident before the kernel
+// ahead of it in the stream has finished (hiding its launch latency); it calls
+// wait_for_prior_kernel() before touching memory.
+template <typename Kernel>
+cudaError_t launch_dependent(Kernel kernel, unsigned grid, unsigned block, size_t smem, cudaStream_t stream, const Params& p) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, p);
+}
+
 cudaError_t launch_merge(const Params& p, cudaStream_t stream) {
   const long long rows = (long long)p.batch * p.M;
-  merge_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, stream>>>(p);
-  return cudaGetLastError();
+  // lanes per row: enough to cover the partial pairs of a row, so that few lanes idle
+  if (p.parts_per_row <= 2) return launch_dependent(merge_kernel<2>, (unsigned)((rows + 127) / 128), 256, 0, stream, p);
+  if (p.parts_per_row <= 16) return launch_dependent(merge_kernel<8>, (unsigned)((rows + 31) / 32), 256, 0, stream, p);
+  return launch_dependent(merge_kernel<32>, (unsigned)((rows + 7) / 8), 256, 0, stream, p);
 }
 
 cudaError_t launch_normalise(const Params& p, cudaStream_t stream) {
   const long long rows = (long long)p.batch * p.M;
   const size_t smem = (size_t)p.parts_per_row * sizeof(float);
-  if (p.dtype == FGR_F32) normalise_kernel<float><<<(unsigned)rows, 256, smem, stream>>>(p);
-  else normalise_kernel<__nv_bfloat16><<<(unsigned)rows, 256, smem, stream>>>(p);
-  return cudaGetLastError();
+  if (p.dtype == FGR_F32) return launch_dependent(normalise_kernel<float>, (unsigned)rows, 256, smem, stream, p);
+  return launch_dependent(normalise_kernel<__nv_bfloat16>, (unsigned)rows, 256, smem, stream, p);
 }
 
 }  // namespace fgr

@@ -328,6 +328,11 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
   if constexpr (PAIR) cluster_sync_all();   // the peer's barriers exist before anything signals them
   tcgen05_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // Programmatic dependent launch: everything above overlapped the tail of the kernel ahead of this
+  // one in the stream; from here on its results (and the workspace it was reading) are needed.  The
+  // merge / normalise kernel that follows may become resident now; it waits for this grid to finish.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if (warp == 0) {
     // ================================================================ TMA producer
@@ -526,23 +531,25 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
 // ------------------------------------------------------------------------------------------ host
 template <int ACT, bool SC, int RED, bool WY>
 cudaError_t launch_one(const Params& p, const CUtensorMap& tx, const CUtensorMap& tw, int grid, int smem, cudaStream_t s) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(kUmmaThreads);
+  cfg.dynamicSmemBytes = (size_t)smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see griddepcontrol in the kernel
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = 2;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
   if (p.cta_pair == 2) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(kUmmaThreads);
-    cfg.dynamicSmemBytes = (size_t)smem;
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, umma_kernel<ACT, SC, RED, WY, true>, tx, tw, p);
   }
-  umma_kernel<ACT, SC, RED, WY, false><<<grid, kUmmaThreads, smem, s>>>(tx, tw, p);
-  return cudaGetLastError();
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, umma_kernel<ACT, SC, RED, WY, false>, tx, tw, p);
 }
 template <int ACT, bool SC, int RED, bool WY>
 cudaError_t prepare_one() {
