@@ -157,12 +157,16 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(const Params p) {
 // them in the stream is still running; this wait returns once that kernel has completed and its
 // writes are visible.  (A no-op for a kernel launched the ordinary way.)
 __device__ __forceinline__ void wait_for_prior_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel in the stream (if it was launched as a programmatic dependent) become
+// resident now and run its set-up; it still waits for this grid to finish before touching memory.
+__device__ __forceinline__ void let_next_kernel_start() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // G lanes per row (32 / G rows per warp): lane t of a group takes partials t, t + G, ... in ascending
 // order, then a fixed xor-shuffle tree combines the G lanes.  The order never depends on timing:
 // bit-identical results from run to run.
 template <int G>
 __global__ void __launch_bounds__(256) merge_kernel(const Params p) {
+  let_next_kernel_start();
   wait_for_prior_kernel();
   const int lane = threadIdx.x & 31, sub = lane % G;
   const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -211,6 +215,7 @@ __global__ void __launch_bounds__(256) merge_kernel(const Params p) {
 template <typename T>
 __global__ void __launch_bounds__(256) normalise_kernel(const Params p) {
   extern __shared__ float factor[];   // [parts_per_row]
+  let_next_kernel_start();
   wait_for_prior_kernel();
   const long long row = blockIdx.x;
   const int bt = (int)(row / p.M), m = (int)(row % p.M);
