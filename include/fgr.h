@@ -91,6 +91,7 @@ typedef struct fgr_desc {
   int32_t force_tile_n;    /* 0 = automatic; else the N extent of a tcgen05 tile (multiple of 16, 16..256) */
   int32_t force_cta_pair;  /* 0 = automatic; 1 = every CTA alone (128-row tiles); 2 = clusters of two CTAs
                               sharing 256-row tiles (tcgen05 cta_group::2; needs tile_n % 32 == 0) */
+  int32_t force_ksub;      /* 0 = automatic; else 1, 2 or 4: 64-wide K sub-blocks per shared-memory ring stage */
 } fgr_desc;
 
 /* What fgr_plan / fgr_create decided; plain host data, for callers, tests and benchmarks. */
@@ -103,6 +104,7 @@ typedef struct fgr_plan_info {
   int32_t launches;        /* kernels launched by one fgr_run */
   int32_t smem_bytes;      /* dynamic shared memory of the main kernel */
   int32_t cta_pair;        /* 2 if the main kernel runs as clusters of two CTAs, else 1 */
+  int32_t ksub;            /* 64-wide K sub-blocks per ring stage (tcgen05 paths; 0 for SIMT) */
   int64_t num_tiles;       /* output tiles in the problem */
   uint64_t workspace_bytes;/* what fgr_run needs */
   double flop;             /* 2 * batch * M * N * K */

@@ -34,14 +34,14 @@ class fgr_desc(ctypes.Structure):
                 ("bsx", ctypes.c_int64), ("bsw", ctypes.c_int64), ("bsy", ctypes.c_int64),
                 ("bias_per_batch", ctypes.c_int32), ("device", ctypes.c_int32),
                 ("force_path", ctypes.c_int32), ("force_tile_n", ctypes.c_int32),
-                ("force_cta_pair", ctypes.c_int32)]
+                ("force_cta_pair", ctypes.c_int32), ("force_ksub", ctypes.c_int32)]
 
 
 class fgr_plan_info(ctypes.Structure):
     _fields_ = [("path", ctypes.c_int32), ("tile_m", ctypes.c_int32), ("tile_n", ctypes.c_int32),
                 ("stages", ctypes.c_int32), ("parts_per_row", ctypes.c_int32), ("grid", ctypes.c_int32),
                 ("launches", ctypes.c_int32), ("smem_bytes", ctypes.c_int32), ("cta_pair", ctypes.c_int32),
-                ("num_tiles", ctypes.c_int64),
+                ("ksub", ctypes.c_int32), ("num_tiles", ctypes.c_int64),
                 ("workspace_bytes", ctypes.c_uint64), ("flop", ctypes.c_double), ("min_bytes", ctypes.c_double)]
 
     def as_dict(self):
@@ -84,9 +84,9 @@ def lib() -> ctypes.CDLL:
 
 
 def make_desc(batch, M, N, K, dtype, act, scale_kind, reduce, *, scale=1.0, write_y=0, ldx=0, ldw=0, ldy=0,
-              bsx=0, bsw=0, bsy=0, bias_per_batch=0, device=0, force_path=FGR_PATH_AUTO, force_tile_n=0, force_cta_pair=0) -> fgr_desc:
+              bsx=0, bsw=0, bsy=0, bias_per_batch=0, device=0, force_path=FGR_PATH_AUTO, force_tile_n=0, force_cta_pair=0, force_ksub=0) -> fgr_desc:
     return fgr_desc(ctypes.sizeof(fgr_desc), batch, M, N, K, dtype, act, scale_kind, reduce, scale, write_y,
-                    ldx, ldw, ldy, bsx, bsw, bsy, bias_per_batch, device, force_path, force_tile_n, force_cta_pair)
+                    ldx, ldw, ldy, bsx, bsw, bsy, bias_per_batch, device, force_path, force_tile_n, force_cta_pair, force_ksub)
 
 
 def fgr_status_string(status: int) -> str:

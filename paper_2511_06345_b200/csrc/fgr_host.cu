@@ -83,6 +83,7 @@ int validate(const fgr_desc* d) {
     return FGR_ERR_INVALID_ARG;
   if ((long long)d->batch * d->M > (1LL << 31) - 1) return FGR_ERR_UNSUPPORTED;
   if (d->force_cta_pair < 0 || d->force_cta_pair > 2) return FGR_ERR_INVALID_ARG;
+  if (d->force_ksub < 0 || d->force_ksub > 4) return FGR_ERR_INVALID_ARG;
   if (d->force_tile_n && (d->force_tile_n % 16 || d->force_tile_n < 16 || d->force_tile_n > 256)) return FGR_ERR_INVALID_ARG;
   return FGR_OK;
 }
@@ -106,7 +107,8 @@ int pick_stream_tile_n(long long tiles_mb, int N, int sms) {
   for (int tn = 16; tn <= 256; tn += 16) {
     const long long tiles = tiles_mb * ((N + tn - 1) / tn);
     const long long waves = (tiles + sms - 1) / sms;
-    const double cost = (double)waves * (tn + 64);
+    // a ragged last tile streams a full X tile for a few real columns: a mild penalty
+    const double cost = (double)waves * (tn + 64) * (N % tn ? 1.1 : 1.0);
     if (cost < best_cost - 1e-9 || (std::fabs(cost - best_cost) <= 1e-9 && tn > best)) { best_cost = cost; best = tn; }
   }
   return best;
@@ -166,11 +168,19 @@ int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
     p.slots_per_tile = 2;
     p.tiles_n = (d.N + tn - 1) / tn;
     const int w_rows = tn / pair;
+    // Two adjacent 64-wide K sub-blocks per ring stage: the memory system then sees requests for
+    // neighbouring 128-byte lines of the same matrix row back to back, which measurably raises the
+    // rate at which operands arrive (L2 and DRAM both work in units larger than one line).  Used
+    // when at least three such stages fit in shared memory and K is long enough to fill them.
+    int ksub = d.force_ksub;
+    if (!ksub) ksub = (d.K > kUmmaBlockK && umma_smem_layout(w_rows, 3, 2).total <= kSmemLimit) ? 2 : 1;
+    while (ksub > 1 && umma_smem_layout(w_rows, 2, ksub).total > kSmemLimit) --ksub;
+    p.ksub = ksub;
     int stages = kUmmaMaxStages;
-    while (stages > 1 && umma_smem_layout(w_rows, stages).total > kSmemLimit) --stages;
+    while (stages > 1 && umma_smem_layout(w_rows, stages, ksub).total > kSmemLimit) --stages;
     p.stages = stages;
     pi.tile_m = kUmmaTileM * pair;
-    pi.smem_bytes = umma_smem_layout(w_rows, stages).total;
+    pi.smem_bytes = umma_smem_layout(w_rows, stages, ksub).total;
   }
   p.num_tiles = (long long)d.batch * p.tiles_m * p.tiles_n;
   p.parts_per_row = p.tiles_n * p.slots_per_tile;
@@ -188,6 +198,7 @@ int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
     pi.grid = (int)(p.num_tiles < groups ? p.num_tiles : groups) * p.cta_pair;
   }
   pi.cta_pair = path == FGR_PATH_SIMT ? 1 : p.cta_pair;
+  pi.ksub = path == FGR_PATH_SIMT ? 0 : p.ksub;
   pi.launches = 2;   // main kernel + (merge | softmax normalise)
   pi.workspace_bytes = (uint64_t)kStatusBytes + (uint64_t)d.batch * d.M * p.parts_per_row * 8ull;
   *info = pi;

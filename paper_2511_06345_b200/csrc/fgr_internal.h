@@ -37,6 +37,7 @@ struct Params {
   int tiles_m, tiles_n;
   long long num_tiles;
   int stages;
+  int ksub;            // tcgen05 paths: 64-wide K sub-blocks per ring stage (1, 2 or 4)
   int cta_pair;        // tcgen05 paths: 1 = each CTA works alone, 2 = clusters of two CTAs share 256-row tiles
 };
 
@@ -49,18 +50,19 @@ __host__ __device__ inline int part_slot(int col, int tile_n, int half_n, int sl
 
 // Shared-memory carve-up of the tcgen05 kernel (offsets from a 1024-byte aligned base).
 struct UmmaSmem {
-  int stage_bytes, x_bytes, w_bytes;
+  int stage_bytes, sub_bytes, x_bytes, w_bytes;   // a stage is `ksub` sub-blocks of (X tile, W tile)
   int vec_off;      // bias / scale staging: [8 epilogue warps][2 vectors][128] floats
   int bar_off;      // mbarriers
   int misc_off;     // TMEM base address, abort flag
   int total;        // bytes to request (includes 1024 of alignment slack)
 };
 // `w_rows`: rows of the W tile one CTA loads per k-block (tile_n, or tile_n / 2 for a CTA pair).
-__host__ __device__ inline UmmaSmem umma_smem_layout(int w_rows, int stages) {
+__host__ __device__ inline UmmaSmem umma_smem_layout(int w_rows, int stages, int ksub) {
   UmmaSmem s;
   s.x_bytes = kUmmaTileM * kUmmaBlockK * 2;
   s.w_bytes = w_rows * kUmmaBlockK * 2;
-  s.stage_bytes = s.x_bytes + s.w_bytes;
+  s.sub_bytes = s.x_bytes + s.w_bytes;
+  s.stage_bytes = s.sub_bytes * ksub;
   s.vec_off = s.stage_bytes * stages;
   s.bar_off = s.vec_off + 8 * 2 * 128 * 4;
   s.misc_off = s.bar_off + (2 * kUmmaMaxStages + 4) * 8;

@@ -287,7 +287,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
   const int w_rows = PAIR ? p.tile_n / 2 : p.tile_n;       // rows of the W tile this CTA loads
-  const UmmaSmem L = umma_smem_layout(w_rows, p.stages);
+  const UmmaSmem L = umma_smem_layout(w_rows, p.stages, p.ksub);
 
   float* vec_s = reinterpret_cast<float*>(base_ptr + L.vec_off);   // [epilogue warp][bias|scale][128]
   const uint32_t bar_base = base + L.bar_off;
@@ -299,7 +299,8 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L.misc_off + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int kblocks = (p.K + kUmmaBlockK - 1) / kUmmaBlockK;
+  const int kstep = kUmmaBlockK * p.ksub;                  // K elements per ring stage
+  const int kblocks = (p.K + kstep - 1) / kstep;
   const int rank = PAIR ? (int)cluster_ctarank() : 0;      // 0 = leader
   // work units are dealt round-robin to CTAs (PAIR: to clusters)
   const long long unit0 = PAIR ? (long long)(blockIdx.x >> 1) : (long long)blockIdx.x;
@@ -348,12 +349,22 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
           const uint32_t xs = base + (uint32_t)(s * L.stage_bytes);
           if constexpr (PAIR) {
             if (rank == 0) mbar_arrive_expect_tx(full_bar(s), 2u * (uint32_t)L.stage_bytes);
-            tma_load_3d_pair(xs, &tmap_x, kb * kUmmaBlockK, c.m0, c.bt, full_bar(s));
-            tma_load_3d_pair(xs + L.x_bytes, &tmap_w, kb * kUmmaBlockK, c.n0 + rank * w_rows, c.bt, full_bar(s));
           } else {
             mbar_arrive_expect_tx(full_bar(s), (uint32_t)L.stage_bytes);
-            tma_load_3d(xs, &tmap_x, kb * kUmmaBlockK, c.m0, c.bt, full_bar(s));
-            tma_load_3d(xs + L.x_bytes, &tmap_w, kb * kUmmaBlockK, c.n0, c.bt, full_bar(s));
+          }
+          // The sub-blocks of a stage are adjacent in K: consecutive requests for the same matrix
+          // rows ask the DRAM for neighbouring 128-byte lines (out-of-range sub-blocks read as zero).
+          for (int j = 0; j < p.ksub; ++j) {
+            const int k0 = kb * kstep + j * kUmmaBlockK;
+            const uint32_t dst = xs + (uint32_t)(j * L.sub_bytes) + L.x_bytes;
+            if constexpr (PAIR) tma_load_3d_pair(dst, &tmap_w, k0, c.n0 + rank * w_rows, c.bt, full_bar(s));
+            else tma_load_3d(dst, &tmap_w, k0, c.n0, c.bt, full_bar(s));
+          }
+          for (int j = 0; j < p.ksub; ++j) {
+            const int k0 = kb * kstep + j * kUmmaBlockK;
+            const uint32_t dst = xs + (uint32_t)(j * L.sub_bytes);
+            if constexpr (PAIR) tma_load_3d_pair(dst, &tmap_x, k0, c.m0, c.bt, full_bar(s));
+            else tma_load_3d(dst, &tmap_x, k0, c.m0, c.bt, full_bar(s));
           }
         }
       }
@@ -387,11 +398,15 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
           if (!(ok = mbar_wait(full_bar(s), ph, abort_flag, p.status))) break;
           tcgen05_fence_after();
           const uint32_t xs = base + (uint32_t)(s * L.stage_bytes);
-          const uint64_t a0 = make_smem_desc(xs), b0 = make_smem_desc(xs + L.x_bytes);
+          for (int j = 0; j < p.ksub; ++j) {
+            const uint64_t a0 = make_smem_desc(xs + (uint32_t)(j * L.sub_bytes));
+            const uint64_t b0 = make_smem_desc(xs + (uint32_t)(j * L.sub_bytes) + L.x_bytes);
 #pragma unroll
-          for (int k = 0; k < kUmmaBlockK / 16; ++k) {   // 16 bf16 = 32 bytes = 2 descriptor address units
-            if constexpr (PAIR) tcgen05_mma_bf16_pair(d, a0 + 2u * k, b0 + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
-            else tcgen05_mma_bf16(d, a0 + 2u * k, b0 + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            for (int k = 0; k < kUmmaBlockK / 16; ++k) {   // 16 bf16 = 32 bytes = 2 descriptor address units
+              const uint32_t acc = (kb | j | k) != 0 ? 1u : 0u;
+              if constexpr (PAIR) tcgen05_mma_bf16_pair(d, a0 + 2u * k, b0 + 2u * k, idesc, acc);
+              else tcgen05_mma_bf16(d, a0 + 2u * k, b0 + 2u * k, idesc, acc);
+            }
           }
           if constexpr (PAIR) tcgen05_commit_pair(empty_bar(s)); else tcgen05_commit(empty_bar(s));
         }

@@ -16,12 +16,12 @@ class FusedGemmReduce:
     """
 
     def __init__(self, batch, M, N, K, dtype, act, scale_kind, reduce, *, scale=1.0, write_y=0, bias_per_batch=0,
-                 device=0, force_path=B.FGR_PATH_AUTO, force_tile_n=0, force_cta_pair=0):
+                 device=0, force_path=B.FGR_PATH_AUTO, force_tile_n=0, force_cta_pair=0, force_ksub=0):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required: this operator has no CPU path")
         self.desc = B.make_desc(batch, M, N, K, dtype, act, scale_kind, reduce, scale=scale, write_y=write_y,
                                 bias_per_batch=bias_per_batch, device=device, force_path=force_path,
-                                force_tile_n=force_tile_n, force_cta_pair=force_cta_pair)
+                                force_tile_n=force_tile_n, force_cta_pair=force_cta_pair, force_ksub=force_ksub)
         self.handle = B.fgr_create(self.desc)
         self.plan = B.fgr_get_plan(self.handle)
         self.device = torch.device("cuda", device)

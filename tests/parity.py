@@ -38,12 +38,12 @@ def to_device(p: gi.Problem, device="cuda:0"):
     return up(p.X, b16), up(p.W, b16), up(p.bias, False), up(p.scale_vec, False)
 
 
-def run_gpu(p: gi.Problem, force_path=0, force_tile_n=0, device=0, tensors=None, repeat=1, force_cta_pair=0):
+def run_gpu(p: gi.Problem, force_path=0, force_tile_n=0, device=0, tensors=None, repeat=1, force_cta_pair=0, force_ksub=0):
     """Runs the operator through fgr_create / fgr_run; returns (Y float64 [rows, N] or None,
     out float64 [rows, w] or None, plan dict)."""
     op = fgr.FusedGemmReduce(p.batch, p.M, p.N, p.K, p.dtype, p.act, p.scale_kind, p.reduce, scale=p.scale,
                              write_y=p.write_y, bias_per_batch=p.bias_per_batch, device=device,
-                             force_path=force_path, force_tile_n=force_tile_n, force_cta_pair=force_cta_pair)
+                             force_path=force_path, force_tile_n=force_tile_n, force_cta_pair=force_cta_pair, force_ksub=force_ksub)
     X, W, b, s = tensors if tensors is not None else to_device(p, "cuda:%d" % device)
     for _ in range(repeat):
         Y, out = op(X, W, b, s)

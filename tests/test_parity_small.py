@@ -110,6 +110,22 @@ def test_cta_pair_and_single_agree_bitwise(cuda_device):
     assert np.array_equal(Y1, Y2) and np.array_equal(o1, o2)
 
 
+def test_k_sub_blocks_per_stage_agree_bitwise(cuda_device):
+    """1, 2 or 4 K sub-blocks per ring stage change how operands are fetched, not what is summed."""
+    for B, M, N, K, tn, pair, path in [(1, 128, 2048, 1096, 112, 1, fgr.FGR_PATH_UMMA_STREAM_W),
+                                       (2, 300, 520, 200, 64, 2, fgr.FGR_PATH_UMMA_TILED),
+                                       (1, 257, 520, 72, 0, 0, fgr.FGR_PATH_UMMA_TILED)]:
+        p = _problem(gi.DTYPE_BF16, B, M, N, K, gi.ACT_GELU_TANH, gi.SCALE_PER_COLUMN, gi.RED_LSE, seed=57)
+        t = to_device(p)
+        ref = None
+        for ks in (1, 2, 4):
+            Y, out, plan = run_gpu(p, tensors=t, force_path=path, force_tile_n=tn, force_cta_pair=pair, force_ksub=ks)
+            if ref is None:
+                compare(p, Y, out)
+                ref = (Y, out)
+            assert np.array_equal(Y, ref[0]) and np.array_equal(out, ref[1]), (B, M, N, K, ks, plan)
+
+
 @pytest.mark.parametrize("red", [gi.RED_LSE, gi.RED_MAXSUM])
 def test_umma_no_y(cuda_device, red):
     p = _problem(gi.DTYPE_BF16, 1, 200, 776, 128, gi.ACT_RELU, gi.SCALE_NONE, red, seed=40, write_y=0)
