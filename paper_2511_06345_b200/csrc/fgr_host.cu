@@ -125,10 +125,11 @@ int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
   int path = d.force_path;
   if (path == FGR_PATH_AUTO) {
     if (d.dtype == FGR_F32) path = FGR_PATH_SIMT;
+    else if (d.M <= 4 && d.reduce != FGR_RED_SOFTMAX) path = FGR_PATH_SIMT_GEMV;   // a few GEMVs: CUDA cores keep up with HBM
     else if (d.M <= 128 && pi.flop / pi.min_bytes < kRidgeFlopPerByte) path = FGR_PATH_UMMA_STREAM_W;
     else path = FGR_PATH_UMMA_TILED;
   }
-  if (path == FGR_PATH_SIMT_GEMV) return FGR_ERR_UNSUPPORTED;   // not built yet
+  if (path == FGR_PATH_SIMT_GEMV && (d.dtype != FGR_BF16 || d.M > 16 || d.reduce == FGR_RED_SOFTMAX)) return FGR_ERR_UNSUPPORTED;
   if ((path == FGR_PATH_UMMA_TILED || path == FGR_PATH_UMMA_STREAM_W) && d.dtype != FGR_BF16) return FGR_ERR_UNSUPPORTED;
 
   Params p;
@@ -138,7 +139,22 @@ int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
   p.write_y = d.write_y; p.bias_per_batch = d.bias_per_batch; p.scale = d.scale;
   p.ldx = r.ldx; p.ldw = r.ldw; p.ldy = r.ldy; p.bsx = r.bsx; p.bsw = r.bsw; p.bsy = r.bsy;
 
-  if (path == FGR_PATH_SIMT) {
+  if (path == FGR_PATH_SIMT_GEMV) {
+    // every CTA streams a contiguous block of W rows; one partial pair per (row of X, CTA)
+    const int r = gemv_rows_per_warp(d.M);
+    int rows = (d.N + sms - 1) / sms;
+    rows = (rows + r - 1) / r * r;
+    p.tile_n = rows;
+    p.half_n = rows;
+    p.slots_per_tile = 1;
+    p.tiles_m = 1;
+    p.tiles_n = (d.N + rows - 1) / rows;
+    p.stages = 0;
+    p.cta_pair = 1;
+    pi.tile_m = d.M;
+    pi.smem_bytes = 0;
+    if (d.batch > 65535) return FGR_ERR_UNSUPPORTED;
+  } else if (path == FGR_PATH_SIMT) {
     p.tile_n = kSimtTile;
     p.half_n = kSimtTile;
     p.slots_per_tile = 1;
@@ -193,12 +209,15 @@ int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
   pi.num_tiles = p.num_tiles;
   if (path == FGR_PATH_SIMT) {
     pi.grid = (int)(p.num_tiles > 0x7fffffff ? 0x7fffffff : p.num_tiles);
+  } else if (path == FGR_PATH_SIMT_GEMV) {
+    pi.grid = p.tiles_n * d.batch;
   } else {
     const long long groups = sms / p.cta_pair;   // CTAs, or clusters of two
     pi.grid = (int)(p.num_tiles < groups ? p.num_tiles : groups) * p.cta_pair;
   }
-  pi.cta_pair = path == FGR_PATH_SIMT ? 1 : p.cta_pair;
-  pi.ksub = path == FGR_PATH_SIMT ? 0 : p.ksub;
+  const bool cuda_cores = path == FGR_PATH_SIMT || path == FGR_PATH_SIMT_GEMV;
+  pi.cta_pair = cuda_cores ? 1 : p.cta_pair;
+  pi.ksub = cuda_cores ? 0 : p.ksub;
   pi.launches = 2;   // main kernel + (merge | softmax normalise)
   pi.workspace_bytes = (uint64_t)kStatusBytes + (uint64_t)d.batch * d.M * p.parts_per_row * 8ull;
   *info = pi;
@@ -336,6 +355,8 @@ int fgr_run(fgr_handle* h, const void* X, const void* W, const float* bias, cons
   if (e == cudaSuccess) {
     if (h->plan.path == FGR_PATH_SIMT) {
       e = launch_simt(p, stream);
+    } else if (h->plan.path == FGR_PATH_SIMT_GEMV) {
+      e = launch_gemv(p, p.tiles_n, p.tile_n, stream);
     } else {
       if (X != h->cached_x) {
         rc = encode_operand(&h->tmap_x, X, d.K, d.M, d.batch, p.ldx, p.bsx, kUmmaTileM);

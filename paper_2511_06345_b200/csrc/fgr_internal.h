@@ -74,6 +74,9 @@ __host__ __device__ inline UmmaSmem umma_smem_layout(int w_rows, int stages, int
 cudaError_t launch_simt(const Params& p, cudaStream_t stream);
 cudaError_t launch_merge(const Params& p, cudaStream_t stream);
 cudaError_t launch_normalise(const Params& p, cudaStream_t stream);
+cudaError_t launch_gemv(const Params& p, int grid, int rows_per_cta, cudaStream_t stream);
+int gemv_rows_per_warp(int M);
+int gemv_k_chunk(int M, int K);
 cudaError_t umma_prepare(int device);   // opt-in shared memory attribute, once per device
 cudaError_t launch_umma(const Params& p, const void* tmap_x, const void* tmap_w, int grid, int smem_bytes,
                         cudaStream_t stream);

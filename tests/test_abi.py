@@ -60,6 +60,10 @@ def test_path_selection_for_the_five_workloads():
     assert c4.stages >= 3 and c4.ksub == 2 and c4.smem_bytes <= 232448
     c5 = _plan(32, 1024, 1024, 512, fgr.FGR_BF16, 1, 0, fgr.FGR_RED_MAXSUM)
     assert c5.path == fgr.FGR_PATH_UMMA_TILED and c5.num_tiles == 512 and c5.cta_pair == 2
+    g = _plan(1, 2, 16384, 8192, fgr.FGR_BF16, 2, 0, fgr.FGR_RED_LSE)          # a few GEMVs: the CUDA-core streaming path
+    assert g.path == fgr.FGR_PATH_SIMT_GEMV and g.grid == g.parts_per_row <= 148 and g.tile_n * g.grid >= 16384
+    assert _plan(1, 2, 16384, 8192, fgr.FGR_BF16, 0, 0, fgr.FGR_RED_SOFTMAX).path == fgr.FGR_PATH_UMMA_STREAM_W
+    assert _plan(1, 8, 16384, 8192, fgr.FGR_BF16, 2, 0, fgr.FGR_RED_LSE).path == fgr.FGR_PATH_UMMA_STREAM_W
     small_sm = fgr.fgr_plan(fgr.make_desc(1, 128, 16384, 8192, fgr.FGR_BF16, 2, 0, 0), 64)
     assert small_sm.grid <= 64
 

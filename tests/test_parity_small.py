@@ -110,6 +110,42 @@ def test_cta_pair_and_single_agree_bitwise(cuda_device):
     assert np.array_equal(Y1, Y2) and np.array_equal(o1, o2)
 
 
+GEMV_SHAPES = [(1, 1, 8, 8), (1, 3, 1000, 264), (1, 8, 2056, 1096), (1, 16, 520, 8200), (3, 5, 264, 72), (1, 2, 4096, 640)]
+
+
+@pytest.mark.parametrize("shape", GEMV_SHAPES)
+@pytest.mark.parametrize("red", [gi.RED_LSE, gi.RED_MAXSUM, gi.RED_MAX_SUMEXP])
+def test_skinny_gemv_path(cuda_device, shape, red):
+    B, M, N, K = shape
+    for i, act in enumerate(ACTS):
+        p = _problem(gi.DTYPE_BF16, B, M, N, K, act, (i + red) % 3, red, seed=60 + i, bias_per_batch=i % 2, write_y=i % 2)
+        Y, out, plan = run_gpu(p, force_path=fgr.FGR_PATH_SIMT_GEMV)
+        assert plan["path"] == fgr.FGR_PATH_SIMT_GEMV and plan["parts_per_row"] == plan["grid"] // B
+        compare(p, Y, out, tcgen05=False)
+
+
+def test_skinny_selection(cuda_device):
+    """M <= 4 goes to the GEMV path by itself; softmax and larger M stay on the tensor-core paths."""
+    assert fgr.fgr_plan(fgr.make_desc(1, 8, 2048, 512, fgr.FGR_BF16, 0, 0, 0)).path == fgr.FGR_PATH_UMMA_STREAM_W
+    p = _problem(gi.DTYPE_BF16, 1, 4, 2048, 512, gi.ACT_GELU_TANH, gi.SCALE_NONE, gi.RED_LSE, seed=63)
+    Y, out, plan = run_gpu(p)
+    assert plan["path"] == fgr.FGR_PATH_SIMT_GEMV
+    compare(p, Y, out, tcgen05=False)
+    ref = out
+    Y, out, plan = run_gpu(p, force_path=fgr.FGR_PATH_UMMA_STREAM_W)      # the same problem on tensor cores
+    compare(p, Y, out)
+    np.testing.assert_allclose(out, ref, rtol=0, atol=2e-4 * (1 + np.abs(ref).max()))
+    p.reduce = gi.RED_SOFTMAX
+    Y, out, plan = run_gpu(p)
+    assert plan["path"] in (fgr.FGR_PATH_UMMA_STREAM_W, fgr.FGR_PATH_UMMA_TILED)
+    compare(p, Y, out)
+    with pytest.raises(fgr.FgrError) as e:
+        fgr.fgr_plan(fgr.make_desc(1, 4, 2048, 512, fgr.FGR_BF16, 0, 0, fgr.FGR_RED_SOFTMAX, force_path=fgr.FGR_PATH_SIMT_GEMV))
+    assert e.value.status == fgr.FGR_ERR_UNSUPPORTED
+    with pytest.raises(fgr.FgrError):
+        fgr.fgr_plan(fgr.make_desc(1, 17, 2048, 512, fgr.FGR_BF16, 0, 0, 0, force_path=fgr.FGR_PATH_SIMT_GEMV))
+
+
 def test_k_sub_blocks_per_stage_agree_bitwise(cuda_device):
     """1, 2 or 4 K sub-blocks per ring stage change how operands are fetched, not what is summed."""
     for B, M, N, K, tn, pair, path in [(1, 128, 2048, 1096, 112, 1, fgr.FGR_PATH_UMMA_STREAM_W),
