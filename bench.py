@@ -350,7 +350,7 @@ def run_ours(args):
 # DRAM bytes per launch of the main kernel from ncu (dram__bytes_read.sum + dram__bytes_write.sum), one
 # capture per workload of the kernel as it stands (profiles/umma_kernel_<workload>.md); a workload
 # without a capture of the current kernel reports null.
-TRAFFIC = {"c2": 85.83e6, "c3": 172.21e6, "c4": 274.65e6, "c5": 73.69e6}
+TRAFFIC = {"c2": 84.17e6, "c3": 171.70e6, "c4": 274.74e6, "c5": 70.83e6}
 
 
 def main():
