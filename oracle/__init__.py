@@ -21,6 +21,7 @@ F32, BF16 = 0, 1
 ACT_NONE, ACT_RELU, ACT_GELU_TANH = 0, 1, 2
 SCALE_NONE, SCALE_SCALAR, SCALE_PER_COLUMN = 0, 1, 2
 RED_LSE, RED_SOFTMAX, RED_MAXSUM, RED_MAX_SUMEXP = 0, 1, 2, 3
+RED_MAX, RED_SUM = 4, 5          # stand-alone reduction only
 
 
 class _Problem(ctypes.Structure):
@@ -50,6 +51,9 @@ def lib() -> ctypes.CDLL:
         _lib.fgr_oracle_rows.restype = ctypes.c_int
         _lib.fgr_oracle_rows.argtypes = [ctypes.POINTER(_Problem)] + [ctypes.c_void_p] * 5 + [
             ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int]
+        _lib.fgr_oracle_reduce_rows.restype = ctypes.c_int
+        _lib.fgr_oracle_reduce_rows.argtypes = [ctypes.c_int32] * 4 + [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
+                                                ctypes.c_void_p]
         _lib.fgr_oracle_gelu_tanh.restype = ctypes.c_double
         _lib.fgr_oracle_gelu_tanh.argtypes = [ctypes.c_double]
         _lib.fgr_oracle_act.restype = ctypes.c_double
@@ -128,3 +132,21 @@ def run_problem(p, rows=None, want_y=True, nthreads=0):
     return run(p.X, p.W, p.bias, p.scale_vec, dtype=p.dtype, act=p.act, scale_kind=p.scale_kind,
                reduce=p.reduce, scale=p.scale, bias_per_batch=p.bias_per_batch, rows=rows, want_y=want_y,
                nthreads=nthreads)
+
+
+def reduce_rows(A, *, dtype, kind):
+    """Reduction over the last dimension of A [M, N] (fp32 values or uint16 bf16 bit patterns; any
+    row stride).  Returns ``(P, out)``: P fp64 [M, N] for SOFTMAX else None; out fp64 [M] (LSE, MAX,
+    SUM), [M, 2] (MAXSUM, MAX_SUMEXP) or None (SOFTMAX)."""
+    want = np.float32 if dtype == F32 else np.uint16
+    if A.dtype != want or A.ndim != 2 or A.strides[1] != A.itemsize:
+        raise TypeError("A must be a 2-D %s array with contiguous rows" % want.__name__)
+    M, N = A.shape
+    lda = A.strides[0] // A.itemsize
+    w = {RED_LSE: 1, RED_SOFTMAX: 0, RED_MAXSUM: 2, RED_MAX_SUMEXP: 2, RED_MAX: 1, RED_SUM: 1}[kind]
+    P = np.empty((M, N), np.float64) if kind == RED_SOFTMAX else None
+    out = np.empty((M, w) if w == 2 else (M,), np.float64) if w else None
+    rc = lib().fgr_oracle_reduce_rows(M, N, dtype, kind, A.ctypes.data_as(ctypes.c_void_p), lda, _ptr(P), _ptr(out))
+    if rc < 0:
+        raise ValueError("fgr_oracle_reduce_rows rejected its arguments (code %d)" % rc)
+    return P, out

@@ -168,3 +168,33 @@ int fgr_oracle_rows(const fgr_oracle_problem* p, const void* X, const void* W, c
 }
 
 int fgr_oracle_out_width(int reduce) { return out_width(reduce); }
+
+/*
+ * Stand-alone reduction over the last dimension of a given matrix A[M, N] (the operator category
+ * "reduction" of Section 4.1, Datasets; the paper's GPU case study is a max reduction over a
+ * dimension, Section 4.4.1).  Same four kinds as above, applied to y = A directly, plus
+ *   kind 4 (MAX): out[m] = max_n A[m, n]          kind 5 (SUM): out[m] = sum_n A[m, n]
+ * P (SOFTMAX) and out are fp64; A is fp32 or bf16 bit patterns, row stride lda elements.
+ * Returns 0, or a negative value on a bad argument.
+ */
+int fgr_oracle_reduce_rows(int32_t M, int32_t N, int32_t dtype, int32_t kind, const void* A, int64_t lda,
+                           double* P, double* out) {
+  if (M < 1 || N < 1 || !A || lda < N) return -1;
+  if (dtype != ORC_F32 && dtype != ORC_BF16) return -3;
+  if (kind < 0 || kind > 5) return -4;
+  for (int64_t m = 0; m < M; ++m) {
+    double mx = load_elem(A, dtype, m * lda);
+    for (int64_t n = 1; n < N; ++n) { double v = load_elem(A, dtype, m * lda + n); if (v > mx) mx = v; }
+    double sum = 0.0, l = 0.0;
+    for (int64_t n = 0; n < N; ++n) { double v = load_elem(A, dtype, m * lda + n); sum += v; l += exp(v - mx); }
+    switch (kind) {
+      case ORC_RED_LSE: out[m] = mx + log(l); break;
+      case ORC_RED_SOFTMAX: for (int64_t n = 0; n < N; ++n) P[m * N + n] = exp(load_elem(A, dtype, m * lda + n) - mx) / l; break;
+      case ORC_RED_MAXSUM: out[2 * m] = mx; out[2 * m + 1] = sum; break;
+      case ORC_RED_MAX_SUMEXP: out[2 * m] = mx; out[2 * m + 1] = l; break;
+      case 4: out[m] = mx; break;
+      default: out[m] = sum; break;
+    }
+  }
+  return 0;
+}

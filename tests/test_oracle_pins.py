@@ -301,3 +301,61 @@ def test_bad_arguments_are_rejected():
         _run(X.astype(np.float64), W, None, None)
     with pytest.raises(ValueError):
         _run(X, _rand((3, 5), 15), None, None)
+
+
+# ---------------------------------------------------------------- stand-alone reduction over rows
+def test_reduce_rows_hand_example():
+    """The y matrix of the hand-computed fixture, reduced directly."""
+    A = _golden("y").reshape(2, 2).astype(np.float32)
+    np.testing.assert_allclose(oracle.reduce_rows(A, dtype=oracle.F32, kind=oracle.RED_LSE)[1], _golden("lse"), atol=1e-14)
+    np.testing.assert_allclose(oracle.reduce_rows(A, dtype=oracle.F32, kind=oracle.RED_SOFTMAX)[0].ravel(), _golden("softmax"), atol=1e-15)
+    np.testing.assert_array_equal(oracle.reduce_rows(A, dtype=oracle.F32, kind=oracle.RED_MAXSUM)[1].ravel(), _golden("maxsum"))
+    np.testing.assert_allclose(oracle.reduce_rows(A, dtype=oracle.F32, kind=oracle.RED_MAX_SUMEXP)[1].ravel(), _golden("max_sumexp"), atol=1e-14)
+    np.testing.assert_array_equal(oracle.reduce_rows(A, dtype=oracle.F32, kind=oracle.RED_MAX)[1], [2, 6])
+    np.testing.assert_array_equal(oracle.reduce_rows(A, dtype=oracle.F32, kind=oracle.RED_SUM)[1], [3, 9])
+
+
+@pytest.mark.parametrize("dtype", [oracle.F32, oracle.BF16])
+def test_reduce_rows_against_library_and_strides(dtype):
+    M, N, lda = 13, 77, 96
+    buf = _rand((M, lda), 31, std=3.0)
+    if dtype == oracle.BF16:
+        bits = gi.f32_to_bf16_bits(buf).reshape(M, lda)
+        A, Af = bits[:, :N], torch.from_numpy(gi.bf16_bits_to_f32(bits).reshape(M, lda)[:, :N].copy()).double()
+    else:
+        A, Af = buf[:, :N], torch.from_numpy(buf[:, :N].copy()).double()
+    assert A.strides[0] == lda * A.itemsize                       # a strided view: the padding must be skipped
+    get = lambda k: oracle.reduce_rows(A, dtype=dtype, kind=k)
+    np.testing.assert_allclose(get(oracle.RED_LSE)[1], torch.logsumexp(Af, 1).numpy(), rtol=1e-13)
+    np.testing.assert_allclose(get(oracle.RED_SOFTMAX)[0], torch.softmax(Af, 1).numpy(), rtol=1e-12)
+    np.testing.assert_array_equal(get(oracle.RED_MAX)[1], Af.amax(1).numpy())
+    np.testing.assert_allclose(get(oracle.RED_SUM)[1], Af.sum(1).numpy(), rtol=0, atol=1e-12)
+    ms = get(oracle.RED_MAXSUM)[1]
+    np.testing.assert_array_equal(ms[:, 0], Af.amax(1).numpy())
+    np.testing.assert_allclose(ms[:, 1], Af.sum(1).numpy(), rtol=0, atol=1e-12)
+    mse = get(oracle.RED_MAX_SUMEXP)[1]
+    np.testing.assert_allclose(mse[:, 0] + np.log(mse[:, 1]), get(oracle.RED_LSE)[1], atol=1e-13)
+
+
+def test_reduce_rows_equals_fused_operator_with_identity_weights():
+    """Reducing A directly = the fused operator with W = I, no bias, no activation, no scale."""
+    n = 40
+    A = _rand((9, n), 32, std=2.0)
+    for kind in (oracle.RED_LSE, oracle.RED_MAXSUM, oracle.RED_MAX_SUMEXP, oracle.RED_SOFTMAX):
+        Y, out, _ = _run(A, np.eye(n, dtype=np.float32), None, None, reduce=kind)
+        P, o = oracle.reduce_rows(A, dtype=oracle.F32, kind=kind)
+        if kind == oracle.RED_SOFTMAX:
+            np.testing.assert_array_equal(P, Y)
+        else:
+            np.testing.assert_array_equal(o.reshape(out.shape), out)
+
+
+def test_reduce_rows_large_magnitudes_and_bad_arguments():
+    A = np.full((2, 16), 900.0, np.float32)           # exp(900) overflows fp64 without the max shift
+    A[1] = -900.0
+    lse = oracle.reduce_rows(A, dtype=oracle.F32, kind=oracle.RED_LSE)[1]
+    np.testing.assert_allclose(lse, [900 + math.log(16), -900 + math.log(16)], rtol=0, atol=1e-12)
+    with pytest.raises(TypeError):
+        oracle.reduce_rows(A.astype(np.float64), dtype=oracle.F32, kind=0)
+    with pytest.raises(KeyError):
+        oracle.reduce_rows(A, dtype=oracle.F32, kind=7)
