@@ -202,6 +202,32 @@ FGR_API int fgr_run_static(const fgr_desc* desc /*host*/, const void* X, const v
                            const float* scale_vec, void* Y, float* out, void* cuda_stream);
 
 /*
+ * fgr_reduce_rows: stand-alone reduction over the last dimension of a given matrix A[M, N] - the
+ * operator category "reduction" (Section 4.1, Datasets); the paper's GPU case study is a max
+ * reduction over a dimension (Section 4.4.1).  The same row reductions as the fused operator,
+ * applied to A itself, plus plain max and plain sum:
+ *     FGR_RED_LSE, FGR_RED_MAXSUM, FGR_RED_MAX_SUMEXP, FGR_REDUCE_MAX, FGR_REDUCE_SUM -> out
+ *     FGR_RED_SOFTMAX -> P[M, N] in A's dtype (P must not overlap A)
+ *   A    device, dtype (fp32 or bf16), row stride lda elements (0 = N), 16-byte aligned, read once
+ *        (twice for softmax, the second time normally from L2)
+ *   P    device, dtype, row stride ldp (0 = N); required iff SOFTMAX
+ *   out  device fp32: [M] (LSE, MAX, SUM) or [M, 2] (MAXSUM, MAX_SUMEXP); required unless SOFTMAX
+ * N, lda and ldp must be multiples of 8 (bf16) / 4 (fp32), else FGR_ERR_UNSUPPORTED.  One kernel
+ * launch on `cuda_stream`, asynchronous, no workspace, no handle; bit-identical from run to run.
+ * Rows are not split across CTAs: the kernel is bandwidth-bound once M is a few hundred or more.
+ */
+enum { FGR_REDUCE_MAX = 4, FGR_REDUCE_SUM = 5 };   /* further values of `reduce` for fgr_reduce_rows only */
+typedef struct fgr_reduce_desc {
+  uint32_t struct_bytes;   /* = sizeof(fgr_reduce_desc) */
+  int32_t M, N;
+  int32_t dtype;           /* fgr_dtype of A and P */
+  int32_t reduce;          /* fgr_reduce, FGR_REDUCE_MAX or FGR_REDUCE_SUM */
+  int32_t device;          /* CUDA device ordinal */
+  int64_t lda, ldp;        /* row strides in elements; 0 = packed */
+} fgr_reduce_desc;
+FGR_API int fgr_reduce_rows(const fgr_reduce_desc* desc /*host*/, const void* A, void* P, float* out, void* cuda_stream);
+
+/*
  * Timing of the main kernel (the GEMM + epilogue + per-tile reduction launch), for benchmarks.
  * fgr_profile_enable(h, 1): from now on fgr_run records a CUDA event before and after its main
  * kernel on the run's stream (at most 4096 runs are kept; later runs are not recorded).

@@ -17,11 +17,12 @@ FGR_F32, FGR_BF16 = 0, 1
 FGR_ACT_NONE, FGR_ACT_RELU, FGR_ACT_GELU_TANH = 0, 1, 2
 FGR_SCALE_NONE, FGR_SCALE_SCALAR, FGR_SCALE_PER_COLUMN = 0, 1, 2
 FGR_RED_LSE, FGR_RED_SOFTMAX, FGR_RED_MAXSUM, FGR_RED_MAX_SUMEXP = 0, 1, 2, 3
+FGR_REDUCE_MAX, FGR_REDUCE_SUM = 4, 5
 FGR_PATH_AUTO, FGR_PATH_SIMT, FGR_PATH_UMMA_TILED, FGR_PATH_UMMA_STREAM_W, FGR_PATH_SIMT_GEMV = 0, 1, 2, 3, 4
 
 FGR_STATIC_SCRATCH_BYTES = 4 << 20
 
-EXPORTS = ("fgr_plan", "fgr_create", "fgr_workspace_bytes", "fgr_get_plan", "fgr_run", "fgr_run_host", "fgr_run_static",
+EXPORTS = ("fgr_plan", "fgr_create", "fgr_workspace_bytes", "fgr_get_plan", "fgr_run", "fgr_run_host", "fgr_run_static", "fgr_reduce_rows",
            "fgr_get_status", "fgr_profile_enable", "fgr_profile_read", "fgr_destroy", "fgr_status_string", "fgr_path_name")
 
 
@@ -35,6 +36,12 @@ class fgr_desc(ctypes.Structure):
                 ("bias_per_batch", ctypes.c_int32), ("device", ctypes.c_int32),
                 ("force_path", ctypes.c_int32), ("force_tile_n", ctypes.c_int32),
                 ("force_cta_pair", ctypes.c_int32), ("force_ksub", ctypes.c_int32)]
+
+
+class fgr_reduce_desc(ctypes.Structure):
+    _fields_ = [("struct_bytes", ctypes.c_uint32), ("M", ctypes.c_int32), ("N", ctypes.c_int32),
+                ("dtype", ctypes.c_int32), ("reduce", ctypes.c_int32), ("device", ctypes.c_int32),
+                ("lda", ctypes.c_int64), ("ldp", ctypes.c_int64)]
 
 
 class fgr_plan_info(ctypes.Structure):
@@ -73,6 +80,7 @@ def lib() -> ctypes.CDLL:
         L.fgr_run.argtypes, L.fgr_run.restype = [vp] * 8 + [ctypes.c_size_t, vp], i
         L.fgr_run_host.argtypes, L.fgr_run_host.restype = [vp] * 7, i
         L.fgr_run_static.argtypes, L.fgr_run_static.restype = [ctypes.POINTER(fgr_desc)] + [vp] * 7, i
+        L.fgr_reduce_rows.argtypes, L.fgr_reduce_rows.restype = [ctypes.POINTER(fgr_reduce_desc)] + [vp] * 4, i
         L.fgr_get_status.argtypes, L.fgr_get_status.restype = [vp], i
         L.fgr_profile_enable.argtypes, L.fgr_profile_enable.restype = [vp, i], i
         L.fgr_profile_read.argtypes, L.fgr_profile_read.restype = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i)], i
@@ -159,6 +167,15 @@ def fgr_run_static(desc: fgr_desc, X, W, bias, scale_vec, Y, out, stream=None, c
                               _addr(out), stream)
     if check and rc != FGR_OK:
         raise FgrError(rc, "fgr_run_static")
+    return rc
+
+
+def fgr_reduce_rows(M, N, dtype, reduce, A, P, out, *, lda=0, ldp=0, device=0, stream=None, check=True) -> int:
+    """Stand-alone reduction over the rows of A [M, N] (device pointers: ints or tensors)."""
+    d = fgr_reduce_desc(ctypes.sizeof(fgr_reduce_desc), M, N, dtype, reduce, device, lda, ldp)
+    rc = lib().fgr_reduce_rows(ctypes.byref(d), _addr(A), _addr(P), _addr(out), stream)
+    if check and rc != FGR_OK:
+        raise FgrError(rc, "fgr_reduce_rows")
     return rc
 
 

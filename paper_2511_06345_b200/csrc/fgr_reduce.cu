@@ -1,0 +1,208 @@
+// Stand-alone reduction over the last dimension of a matrix A[M, N]: max, sum, (max, sum),
+// LogSumExp, (max, sum-exp) and softmax.  HBM-bound: every element is read once with 128-bit loads
+// (softmax reads the row a second time, normally from L2, and writes P once).  G threads share a
+// row (a warp for short rows, a whole CTA for long ones); each thread keeps an online
+// (max, sum of 2^((v - max) log2 e)) pair and a plain sum, and a fixed shuffle / shared-memory tree
+// combines them, so results repeat bit for bit.
+#include <cuda_bf16.h>
+#include <math_constants.h>
+
+#include "fgr.h"
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct ReduceParams {
+  int M, N, kind;
+  long long lda, ldp;
+  const void* A;
+  void* P;
+  float* out;
+};
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+template <typename T> struct Vec;
+template <> struct Vec<float> {
+  static constexpr int kElems = 4;
+  __device__ static void load(const float* p, float* v) {
+    const float4 r = *reinterpret_cast<const float4*>(p);
+    v[0] = r.x; v[1] = r.y; v[2] = r.z; v[3] = r.w;
+  }
+  __device__ static void store(float* p, const float* v) { *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]); }
+};
+template <> struct Vec<__nv_bfloat16> {
+  static constexpr int kElems = 8;
+  __device__ static void load(const __nv_bfloat16* p, float* v) {
+    const uint4 r = *reinterpret_cast<const uint4*>(p);
+    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { v[2 * i] = __uint_as_float(w[i] << 16); v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u); }
+  }
+  __device__ static void store(__nv_bfloat16* p, const float* v) {
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+      w[i] = *reinterpret_cast<uint32_t*>(&h);
+    }
+    *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+};
+
+struct State { float m, l, s; };   // max, sum of 2^((v - max) log2 e), plain sum
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {   // x + y on one lane, y + x on its partner: the same bits
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+// All lanes of a warp end up with the warp's (max, sum-exp relative to that max, sum).
+template <bool EXP>
+__device__ __forceinline__ State warp_combine(State st) {
+  const float m = warp_max(st.m);
+  if (EXP) st.l = warp_sum(st.m > -CUDART_INF_F ? st.l * ex2((st.m - m) * kLog2e) : 0.0f);
+  st.m = m;
+  st.s = warp_sum(st.s);
+  return st;
+}
+
+// G = threads per row: 32 (a warp, kThreads / 32 rows per CTA) or kThreads (one row per CTA).
+template <typename T, int G, bool EXP>
+__global__ void __launch_bounds__(kThreads) reduce_rows_kernel(const ReduceParams p) {
+  constexpr int V = Vec<T>::kElems;
+  constexpr int kRowsPerCta = kThreads / G;
+  __shared__ State red[kThreads / 32];
+  const int sub = threadIdx.x % G;
+  const long long row = (long long)blockIdx.x * kRowsPerCta + threadIdx.x / G;
+  const bool row_ok = row < p.M;
+  const T* a = static_cast<const T*>(p.A) + (row_ok ? row : 0) * p.lda;
+
+  State st = {-CUDART_INF_F, 0.0f, 0.0f};
+  if (row_ok) {
+    // four vectors per thread and iteration: four independent 128-bit loads in flight
+    for (int c0 = sub * V; c0 < p.N; c0 += 4 * G * V) {
+      float v[4][V];
+      int nv = 0;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int c = c0 + u * G * V;
+        if (c < p.N) { Vec<T>::load(a + c, v[u]); nv = u + 1; }
+      }
+      float vm = -CUDART_INF_F;
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (u < nv) {
+#pragma unroll
+          for (int j = 0; j < V; ++j) { vm = fmaxf(vm, v[u][j]); st.s += v[u][j]; }
+        }
+      if (EXP) {
+        const float mn = fmaxf(st.m, vm);
+        float l = 0.0f;
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (u < nv) {
+#pragma unroll
+            for (int j = 0; j < V; ++j) l += ex2((v[u][j] - mn) * kLog2e);
+          }
+        st.l = st.l * ex2((st.m - mn) * kLog2e) + l;
+        st.m = mn;
+      } else {
+        st.m = fmaxf(st.m, vm);
+      }
+    }
+  }
+  // combine the threads of a row: inside the warp by shuffles ...
+  st = warp_combine<EXP>(st);
+  // ... then, for a row spread over the whole CTA, the warps in warp order
+  if (G == kThreads) {
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = st;
+    __syncthreads();
+    float m = red[0].m;
+#pragma unroll
+    for (int w = 1; w < kThreads / 32; ++w) m = fmaxf(m, red[w].m);
+    float l = 0.0f, sum = 0.0f;
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) {
+      if (EXP) l += red[w].m > -CUDART_INF_F ? red[w].l * ex2((red[w].m - m) * kLog2e) : 0.0f;
+      sum += red[w].s;
+    }
+    st.m = m; st.l = l; st.s = sum;
+  }
+  if (!row_ok) return;
+  if (sub == 0) {
+    switch (p.kind) {
+      case FGR_RED_LSE: p.out[row] = st.m + logf(st.l); break;
+      case FGR_RED_MAXSUM: reinterpret_cast<float2*>(p.out)[row] = make_float2(st.m, st.s); break;
+      case FGR_RED_MAX_SUMEXP: reinterpret_cast<float2*>(p.out)[row] = make_float2(st.m, st.l); break;
+      case FGR_REDUCE_MAX: p.out[row] = st.m; break;
+      case FGR_REDUCE_SUM: p.out[row] = st.s; break;
+      default: break;
+    }
+  }
+  if (p.kind == FGR_RED_SOFTMAX) {
+    // second pass: the row was read a moment ago, so it normally comes from L2
+    T* dst = static_cast<T*>(p.P) + row * p.ldp;
+    const float inv = 1.0f / st.l;
+    for (int c = sub * V; c < p.N; c += G * V) {
+      float v[V];
+      Vec<T>::load(a + c, v);
+#pragma unroll
+      for (int j = 0; j < V; ++j) v[j] = ex2((v[j] - st.m) * kLog2e) * inv;
+      Vec<T>::store(dst + c, v);
+    }
+  }
+}
+
+template <typename T>
+cudaError_t launch(const ReduceParams& p, cudaStream_t s) {
+  const bool exp_kind = p.kind == FGR_RED_LSE || p.kind == FGR_RED_SOFTMAX || p.kind == FGR_RED_MAX_SUMEXP;
+  const bool warp_rows = p.N <= 32 * Vec<T>::kElems * 8;   // a warp covers the row in at most two iterations
+  const unsigned grid = warp_rows ? (unsigned)((p.M + kThreads / 32 - 1) / (kThreads / 32)) : (unsigned)p.M;
+  if (warp_rows) {
+    if (exp_kind) reduce_rows_kernel<T, 32, true><<<grid, kThreads, 0, s>>>(p);
+    else reduce_rows_kernel<T, 32, false><<<grid, kThreads, 0, s>>>(p);
+  } else {
+    if (exp_kind) reduce_rows_kernel<T, kThreads, true><<<grid, kThreads, 0, s>>>(p);
+    else reduce_rows_kernel<T, kThreads, false><<<grid, kThreads, 0, s>>>(p);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+extern "C" int fgr_reduce_rows(const fgr_reduce_desc* d, const void* A, void* P, float* out, void* cuda_stream) {
+  if (!d || d->struct_bytes != sizeof(fgr_reduce_desc) || !A) return FGR_ERR_INVALID_ARG;
+  if (d->dtype != FGR_F32 && d->dtype != FGR_BF16) return FGR_ERR_INVALID_ARG;
+  if (d->reduce < FGR_RED_LSE || d->reduce > FGR_REDUCE_SUM) return FGR_ERR_INVALID_ARG;
+  if (d->M < 1 || d->N < 1 || d->device < 0 || d->lda < 0 || d->ldp < 0) return FGR_ERR_INVALID_ARG;
+  const int g = d->dtype == FGR_F32 ? 4 : 8;   // elements per 16 bytes
+  const long long lda = d->lda ? d->lda : d->N, ldp = d->ldp ? d->ldp : d->N;
+  if (lda < d->N || ldp < d->N) return FGR_ERR_INVALID_ARG;
+  if (d->N % g || lda % g || ldp % g) return FGR_ERR_UNSUPPORTED;
+  const bool softmax = d->reduce == FGR_RED_SOFTMAX;
+  if (softmax ? !P : !out) return FGR_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(A) & 15u) || (softmax && (reinterpret_cast<uintptr_t>(P) & 15u)) ||
+      (out && (reinterpret_cast<uintptr_t>(out) & 7u)))
+    return FGR_ERR_INVALID_ARG;
+  int prev = -1;
+  cudaGetDevice(&prev);
+  if (prev != d->device && cudaSetDevice(d->device) != cudaSuccess) { cudaGetLastError(); return FGR_ERR_CUDA; }
+  ReduceParams p = {d->M, d->N, d->reduce, lda, ldp, A, P, out};
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e = d->dtype == FGR_F32 ? launch<float>(p, s) : launch<__nv_bfloat16>(p, s);
+  if (prev != d->device && prev >= 0) cudaSetDevice(prev);
+  if (e != cudaSuccess) { cudaGetLastError(); return FGR_ERR_CUDA; }
+  return FGR_OK;
+}
