@@ -31,16 +31,14 @@ __device__ __forceinline__ float ex2(float x) {
 template <typename T> struct Vec;
 template <> struct Vec<float> {
   static constexpr int kElems = 4;
-  __device__ static void load(const float* p, float* v) {
-    const float4 r = *reinterpret_cast<const float4*>(p);
-    v[0] = r.x; v[1] = r.y; v[2] = r.z; v[3] = r.w;
+  __device__ static void unpack(const uint4& r, float* v) {
+    v[0] = __uint_as_float(r.x); v[1] = __uint_as_float(r.y); v[2] = __uint_as_float(r.z); v[3] = __uint_as_float(r.w);
   }
   __device__ static void store(float* p, const float* v) { *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]); }
 };
 template <> struct Vec<__nv_bfloat16> {
   static constexpr int kElems = 8;
-  __device__ static void load(const __nv_bfloat16* p, float* v) {
-    const uint4 r = *reinterpret_cast<const uint4*>(p);
+  __device__ static void unpack(const uint4& r, float* v) {
     const uint32_t w[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) { v[2 * i] = __uint_as_float(w[i] << 16); v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u); }
@@ -69,18 +67,19 @@ __device__ __forceinline__ float warp_sum(float v) {   // x + y on one lane, y +
   return v;
 }
 // All lanes of a warp end up with the warp's (max, sum-exp relative to that max, sum).
-template <bool EXP>
+template <bool EXP, bool SUM>
 __device__ __forceinline__ State warp_combine(State st) {
   const float m = warp_max(st.m);
   if (EXP) st.l = warp_sum(st.m > -CUDART_INF_F ? st.l * ex2((st.m - m) * kLog2e) : 0.0f);
   st.m = m;
-  st.s = warp_sum(st.s);
+  if (SUM) st.s = warp_sum(st.s);
   return st;
 }
 
 // G = threads per row: 32 (a warp, kThreads / 32 rows per CTA) or kThreads (one row per CTA).
-template <typename T, int G, bool EXP>
-__global__ void __launch_bounds__(kThreads) reduce_rows_kernel(const ReduceParams p) {
+// EXP: the kind needs sum-exp; SUM: it needs the plain sum.
+template <typename T, int G, bool EXP, bool SUM>
+__global__ void __launch_bounds__(kThreads, 8) reduce_rows_kernel(const ReduceParams p) {
   constexpr int V = Vec<T>::kElems;
   constexpr int kRowsPerCta = kThreads / G;
   __shared__ State red[kThreads / 32];
@@ -91,30 +90,37 @@ __global__ void __launch_bounds__(kThreads) reduce_rows_kernel(const ReduceParam
 
   State st = {-CUDART_INF_F, 0.0f, 0.0f};
   if (row_ok) {
-    // four vectors per thread and iteration: four independent 128-bit loads in flight
+    // four vectors per thread and iteration: four independent 128-bit loads in flight.  The raw
+    // 16-byte words are kept and unpacked where they are used (twice for the exp kinds): that keeps
+    // the register count low enough for eight CTAs per SM, i.e. for enough bytes in flight.
     for (int c0 = sub * V; c0 < p.N; c0 += 4 * G * V) {
-      float v[4][V];
+      uint4 raw[4];
       int nv = 0;
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int c = c0 + u * G * V;
-        if (c < p.N) { Vec<T>::load(a + c, v[u]); nv = u + 1; }
+        if (c < p.N) { raw[u] = *reinterpret_cast<const uint4*>(a + c); nv = u + 1; }
       }
       float vm = -CUDART_INF_F;
 #pragma unroll
       for (int u = 0; u < 4; ++u)
         if (u < nv) {
+          float v[V];
+          Vec<T>::unpack(raw[u], v);
 #pragma unroll
-          for (int j = 0; j < V; ++j) { vm = fmaxf(vm, v[u][j]); st.s += v[u][j]; }
+          for (int j = 0; j < V; ++j) { vm = fmaxf(vm, v[j]); if (SUM) st.s += v[j]; }
         }
       if (EXP) {
         const float mn = fmaxf(st.m, vm);
+        const float off = mn * kLog2e;
         float l = 0.0f;
 #pragma unroll
         for (int u = 0; u < 4; ++u)
           if (u < nv) {
+            float v[V];
+            Vec<T>::unpack(raw[u], v);
 #pragma unroll
-            for (int j = 0; j < V; ++j) l += ex2((v[u][j] - mn) * kLog2e);
+            for (int j = 0; j < V; ++j) l += ex2(fmaf(v[j], kLog2e, -off));
           }
         st.l = st.l * ex2((st.m - mn) * kLog2e) + l;
         st.m = mn;
@@ -124,7 +130,7 @@ __global__ void __launch_bounds__(kThreads) reduce_rows_kernel(const ReduceParam
     }
   }
   // combine the threads of a row: inside the warp by shuffles ...
-  st = warp_combine<EXP>(st);
+  st = warp_combine<EXP, SUM>(st);
   // ... then, for a row spread over the whole CTA, the warps in warp order
   if (G == kThreads) {
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = st;
@@ -157,7 +163,7 @@ __global__ void __launch_bounds__(kThreads) reduce_rows_kernel(const ReduceParam
     const float inv = 1.0f / st.l;
     for (int c = sub * V; c < p.N; c += G * V) {
       float v[V];
-      Vec<T>::load(a + c, v);
+      Vec<T>::unpack(*reinterpret_cast<const uint4*>(a + c), v);
 #pragma unroll
       for (int j = 0; j < V; ++j) v[j] = ex2((v[j] - st.m) * kLog2e) * inv;
       Vec<T>::store(dst + c, v);
@@ -170,13 +176,16 @@ cudaError_t launch(const ReduceParams& p, cudaStream_t s) {
   const bool exp_kind = p.kind == FGR_RED_LSE || p.kind == FGR_RED_SOFTMAX || p.kind == FGR_RED_MAX_SUMEXP;
   const bool warp_rows = p.N <= 32 * Vec<T>::kElems * 8;   // a warp covers the row in at most two iterations
   const unsigned grid = warp_rows ? (unsigned)((p.M + kThreads / 32 - 1) / (kThreads / 32)) : (unsigned)p.M;
-  if (warp_rows) {
-    if (exp_kind) reduce_rows_kernel<T, 32, true><<<grid, kThreads, 0, s>>>(p);
-    else reduce_rows_kernel<T, 32, false><<<grid, kThreads, 0, s>>>(p);
-  } else {
-    if (exp_kind) reduce_rows_kernel<T, kThreads, true><<<grid, kThreads, 0, s>>>(p);
-    else reduce_rows_kernel<T, kThreads, false><<<grid, kThreads, 0, s>>>(p);
-  }
+  const bool sum_kind = p.kind == FGR_RED_MAXSUM || p.kind == FGR_REDUCE_SUM;
+#define FGR_REDUCE_LAUNCH(Gv) \
+  do { \
+    if (exp_kind) reduce_rows_kernel<T, Gv, true, false><<<grid, kThreads, 0, s>>>(p); \
+    else if (sum_kind) reduce_rows_kernel<T, Gv, false, true><<<grid, kThreads, 0, s>>>(p); \
+    else reduce_rows_kernel<T, Gv, false, false><<<grid, kThreads, 0, s>>>(p); \
+  } while (0)
+  if (warp_rows) FGR_REDUCE_LAUNCH(32);
+  else FGR_REDUCE_LAUNCH(kThreads);
+#undef FGR_REDUCE_LAUNCH
   return cudaGetLastError();
 }
 
