@@ -347,6 +347,98 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+REDUCE_CONFIGS = {   # stand-alone row reduction of a bf16 matrix, the paper's GPU case-study category (Section 4.4.1)
+    "r_max": dict(M=8192, N=8192, kind=4, name="max"),
+    "r_lse": dict(M=8192, N=8192, kind=0, name="lse"),
+    "r_softmax": dict(M=8192, N=8192, kind=1, name="softmax"),
+}
+
+
+def run_reduce(args):
+    """Bench leg of fgr_reduce_rows: same JSON contract; one step = one launch over one matrix."""
+    import numpy as np
+    import torch
+    import fgr_inputs as gi
+    import paper_2511_06345_b200 as fgr
+    rank, local_rank, world = dist_env()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    c = REDUCE_CONFIGS[args.config]
+    M, N, kind = c["M"], c["N"], c["kind"]
+    peaks, peak_src = load_peaks()
+    rot = 3                                                    # 3 x 134 MB > 126 MB L2
+    hosts = [gi.f32_to_bf16_bits(gi.normal(1000 * rank + r, 9, M * N, 2.0)).reshape(M, N) for r in range(rot)]
+    mats = [torch.from_numpy(h).view(torch.int16).view(torch.bfloat16).to(dev) for h in hosts]
+    P = torch.empty((M, N), dtype=torch.bfloat16, device=dev) if kind == 1 else None
+    out = None if kind == 1 else torch.empty((M, 2), dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream(dev).cuda_stream
+    step = lambda i: fgr.fgr_reduce_rows(M, N, fgr.FGR_BF16, kind, mats[i % rot], P, out, device=local_rank, stream=stream)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize(dev)
+    t1 = time.perf_counter()
+    sampler.stop()
+    ms_step = max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps
+    nbytes = M * N * 2 * (2 if kind == 1 else 1) + (0 if kind == 1 else M * 4)
+    value = world * nbytes / (ms_step * 1e-3) / 1e9
+    # end to end: pinned host matrix in, result out, around the same C-ABI call
+    hp = torch.from_numpy(hosts[0]).pin_memory()
+    res_h = torch.empty((M, N), dtype=torch.int16).pin_memory() if kind == 1 else torch.empty((M, 2), dtype=torch.float32).pin_memory()
+    stage = mats[0]
+    e2e_steps = max(3, min(args.steps, 20))
+    def e2e_step():
+        stage.view(torch.int16).copy_(hp.view(torch.int16), non_blocking=True)
+        fgr.fgr_reduce_rows(M, N, fgr.FGR_BF16, kind, stage, P, out, device=local_rank, stream=stream)
+        (res_h.copy_(P.view(torch.int16), non_blocking=True) if kind == 1 else res_h.copy_(out, non_blocking=True))
+        torch.cuda.synchronize(dev)
+    e2e_step()
+    te = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    dt = max_over_ranks((time.perf_counter() - te) / e2e_steps, world, dev)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        rows = 512
+        tc = time.perf_counter()
+        oracle.reduce_rows(hosts[0][:rows], dtype=oracle.BF16, kind=kind)
+        dtc = time.perf_counter() - tc
+        cpu = {"value": nbytes * rows / M / dtc / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle", "seconds": dtc,
+               "sample": "the first %d of %d rows, fp64 loops, one thread" % (rows, M)}
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+                "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+                "data": "synthetic", "config": {"workload": args.config, "M": M, "N": N, "reduce": c["name"],
+                "l2": "rotating %d distinct matrices (%.0f MB > 126 MB L2)" % (rot, rot * M * N * 2 / 1e6)},
+                "clocks": sampler.summary(t0, t1), "gpu_launches": args.steps,
+                "roofline": {"bound": "hbm", "achieved": value / world, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                             "frac": value / world / peaks["hbm_gbs"], "peak_source": peak_src, "kernel": "reduce_rows_kernel",
+                             "kernel_us": ms_step * 1e3, "timing": "the step is this one kernel", "traffic": None},
+                "e2e": {"value": world * nbytes / dt / 1e9, "unit": "GB/s", "h2d_bytes_per_step": M * N * 2,
+                        "d2h_bytes_per_step": res_h.numel() * res_h.element_size(), "steps": e2e_steps, "ms_per_step": dt * 1e3}}
+        if cpu:
+            line["cpu_baseline"] = cpu
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 # DRAM bytes per launch of the main kernel from ncu (dram__bytes_read.sum + dram__bytes_write.sum), one
 # capture per workload of the kernel as it stands (profiles/umma_kernel_<workload>.md); a workload
 # without a capture of the current kernel reports null.
@@ -359,11 +451,15 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5"] + sorted(REDUCE_CONFIGS))
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.config in REDUCE_CONFIGS:
+        if args.impl == "reference":
+            raise SystemExit("the reference arm covers the fused operator's workloads c1..c5")
+        run_reduce(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
