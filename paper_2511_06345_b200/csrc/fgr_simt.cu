@@ -77,16 +77,23 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(const Params p) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
 
-  for (int k0 = 0; k0 < p.K; k0 += BK) {
-    float4 xv = make_float4(0.f, 0.f, 0.f, 0.f), wv = xv;
+  // the loads of k-block i + 1 are issued before the FMAs of k-block i, so their latency is hidden
+  auto fetch = [&](int k0, float4& xv, float4& wv) {
+    xv = make_float4(0.f, 0.f, 0.f, 0.f);
+    wv = xv;
     if (k0 + lk < p.K) {   // K is a multiple of 4: the four elements are in range together
       if (m0 + lr < p.M) xv = load4(X + (long long)(m0 + lr) * p.ldx + k0 + lk);
       if (n0 + lr < p.N) wv = load4(W + (long long)(n0 + lr) * p.ldw + k0 + lk);
     }
+  };
+  float4 xv, wv;
+  fetch(0, xv, wv);
+  for (int k0 = 0; k0 < p.K; k0 += BK) {
     __syncthreads();
     Xs[lk + 0][lr] = xv.x; Xs[lk + 1][lr] = xv.y; Xs[lk + 2][lr] = xv.z; Xs[lk + 3][lr] = xv.w;
     Ws[lk + 0][lr] = wv.x; Ws[lk + 1][lr] = wv.y; Ws[lk + 2][lr] = wv.z; Ws[lk + 3][lr] = wv.w;
     __syncthreads();
+    if (k0 + BK < p.K) fetch(k0 + BK, xv, wv);
 #pragma unroll
     for (int k = 0; k < BK; ++k) {
       float4 a = *reinterpret_cast<const float4*>(&Xs[k][ty * 4]);
