@@ -36,7 +36,7 @@ TENSOR_X, TENSOR_W, TENSOR_BIAS, TENSOR_SCALE = 1, 2, 3, 4
 
 # enum values of the operator descriptor (documented in include/fgr.h)
 DTYPE_F32, DTYPE_BF16 = 0, 1
-ACT_NONE, ACT_RELU, ACT_GELU_TANH = 0, 1, 2
+ACT_NONE, ACT_RELU, ACT_GELU_TANH, ACT_SIGMOID, ACT_TANH, ACT_SILU = 0, 1, 2, 3, 4, 5
 SCALE_NONE, SCALE_SCALAR, SCALE_PER_COLUMN = 0, 1, 2
 RED_LSE, RED_SOFTMAX, RED_MAXSUM, RED_MAX_SUMEXP = 0, 1, 2, 3
 

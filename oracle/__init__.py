@@ -18,7 +18,7 @@ _SRC = os.path.join(_HERE, "fgr_oracle.c")
 _LIB = os.path.join(_HERE, "libfgr_oracle.so")
 
 F32, BF16 = 0, 1
-ACT_NONE, ACT_RELU, ACT_GELU_TANH = 0, 1, 2
+ACT_NONE, ACT_RELU, ACT_GELU_TANH, ACT_SIGMOID, ACT_TANH, ACT_SILU = 0, 1, 2, 3, 4, 5
 SCALE_NONE, SCALE_SCALAR, SCALE_PER_COLUMN = 0, 1, 2
 RED_LSE, RED_SOFTMAX, RED_MAXSUM, RED_MAX_SUMEXP = 0, 1, 2, 3
 RED_MAX, RED_SUM = 4, 5          # stand-alone reduction only

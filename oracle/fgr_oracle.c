@@ -25,6 +25,7 @@
  *
  *   act: NONE a = u;  RELU a = max(u, 0);
  *        GELU_TANH a = 0.5 u (1 + tanh( sqrt(2/pi) (u + 0.044715 u^3) ))
+ *        SIGMOID a = 1 / (1 + e^-u);  TANH a = tanh u;  SILU a = u / (1 + e^-u)
  *
  * Inputs are the very bits the GPU gets: fp32 values, or bf16 bit patterns
  * (uint16) that are widened exactly to fp64 here.  Rows are independent; the
@@ -46,7 +47,7 @@
 #endif
 
 enum { ORC_F32 = 0, ORC_BF16 = 1 };
-enum { ORC_ACT_NONE = 0, ORC_ACT_RELU = 1, ORC_ACT_GELU_TANH = 2 };
+enum { ORC_ACT_NONE = 0, ORC_ACT_RELU = 1, ORC_ACT_GELU_TANH = 2, ORC_ACT_SIGMOID = 3, ORC_ACT_TANH = 4, ORC_ACT_SILU = 5 };
 enum { ORC_SCALE_NONE = 0, ORC_SCALE_SCALAR = 1, ORC_SCALE_PER_COLUMN = 2 };
 enum { ORC_RED_LSE = 0, ORC_RED_SOFTMAX = 1, ORC_RED_MAXSUM = 2, ORC_RED_MAX_SUMEXP = 3 };
 
@@ -80,6 +81,9 @@ double fgr_oracle_act(int act, double u) {
   switch (act) {
     case ORC_ACT_RELU: return u > 0.0 ? u : 0.0;
     case ORC_ACT_GELU_TANH: return fgr_oracle_gelu_tanh(u);
+    case ORC_ACT_SIGMOID: return 1.0 / (1.0 + exp(-u));          /* logistic function */
+    case ORC_ACT_TANH: return tanh(u);
+    case ORC_ACT_SILU: return u / (1.0 + exp(-u));             /* u * sigmoid(u) */
     default: return u;
   }
 }
@@ -135,7 +139,7 @@ int fgr_oracle_rows(const fgr_oracle_problem* p, const void* X, const void* W, c
   if (!p || !X || !W || nrows < 0) return -1;
   if (p->batch < 1 || p->M < 1 || p->N < 1 || p->K < 1) return -2;
   if (p->dtype != ORC_F32 && p->dtype != ORC_BF16) return -3;
-  if (p->act < 0 || p->act > 2 || p->scale_kind < 0 || p->scale_kind > 2 || p->reduce < 0 || p->reduce > 3) return -4;
+  if (p->act < 0 || p->act > 5 || p->scale_kind < 0 || p->scale_kind > 2 || p->reduce < 0 || p->reduce > 3) return -4;
   if (p->scale_kind == ORC_SCALE_PER_COLUMN && !scale_vec) return -5;
   const int64_t total = (int64_t)p->batch * p->M;
   for (int64_t i = 0; i < nrows; ++i) {

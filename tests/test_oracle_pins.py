@@ -359,3 +359,34 @@ def test_reduce_rows_large_magnitudes_and_bad_arguments():
         oracle.reduce_rows(A.astype(np.float64), dtype=oracle.F32, kind=0)
     with pytest.raises(KeyError):
         oracle.reduce_rows(A, dtype=oracle.F32, kind=7)
+
+
+# ---------------------------------------------------------------- further activations
+def test_sigmoid_tanh_silu_closed_forms_and_library():
+    sg = lambda x: oracle.act(oracle.ACT_SIGMOID, x)
+    th = lambda x: oracle.act(oracle.ACT_TANH, x)
+    si = lambda x: oracle.act(oracle.ACT_SILU, x)
+    assert sg(0.0) == 0.5 and th(0.0) == 0.0 and si(0.0) == 0.0
+    assert sg(1.0) == pytest.approx(0.7310585786300049, abs=1e-16)      # 1 / (1 + e^-1), tabulated
+    assert th(1.0) == pytest.approx(0.7615941559557649, abs=1e-16)      # tanh 1, tabulated
+    for x in [0.01, 0.3, 1.0, 2.5, 9.0]:
+        assert sg(x) + sg(-x) == pytest.approx(1.0, abs=1e-15)           # logistic symmetry
+        assert th(x) == -th(-x)                                          # odd
+        assert th(x) == pytest.approx(2 * sg(2 * x) - 1, abs=1e-15)      # tanh x = 2 sigmoid(2x) - 1
+        assert si(x) == pytest.approx(x * sg(x), rel=1e-15)              # SiLU = x sigmoid(x)
+        assert si(x) - si(-x) == pytest.approx(x, rel=1e-14)
+    assert sg(40.0) == pytest.approx(1.0, abs=1e-15) and sg(-745.0) >= 0.0 and th(20.0) == 1.0
+    xs = torch.linspace(-8, 8, 65, dtype=torch.float64)
+    for kind, fn in [(oracle.ACT_SIGMOID, torch.sigmoid), (oracle.ACT_TANH, torch.tanh), (oracle.ACT_SILU, torch.nn.functional.silu)]:
+        got = np.array([oracle.act(kind, float(x)) for x in xs])
+        np.testing.assert_allclose(got, fn(xs).numpy(), rtol=0, atol=2e-15)
+
+
+@pytest.mark.parametrize("act,fn", [(oracle.ACT_SIGMOID, torch.sigmoid), (oracle.ACT_TANH, torch.tanh),
+                                    (oracle.ACT_SILU, torch.nn.functional.silu)])
+def test_further_activations_in_the_chain(act, fn):
+    X, W, b = _rand((6, 10), 41, std=1.5), _rand((14, 10), 41, tid=8, std=1.5), gi.uniform(41, 3, 14, -1, 1)
+    Y, out, _ = _run(X, W, b, None, act=act, scale_kind=oracle.SCALE_SCALAR, scale=-0.5, reduce=oracle.RED_LSE)
+    y = fn(torch.from_numpy(X).double() @ torch.from_numpy(W).double().T + torch.from_numpy(b).double()) * -0.5
+    np.testing.assert_allclose(Y, y.numpy(), rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(out[:, 0], torch.logsumexp(y, 1).numpy(), rtol=1e-13)
