@@ -4,7 +4,7 @@
  * The operator.  For every batch bt and row m
  *
  *     z[m, n] = sum_k X[bt, m, k] * W[bt, n, k]            (X * W^T, K contiguous in both)
- *     y[m, n] = act(z[m, n] + b[n]) * s[n]                  act in {identity, ReLU, GELU-tanh}
+ *     y[m, n] = act(z[m, n] + b[n]) * s[n]                  act in {identity, ReLU, GELU-tanh, sigmoid, tanh, SiLU}
  *
  * followed by a reduction over n of each row:
  *
@@ -61,7 +61,8 @@ typedef enum {
 } fgr_status;
 
 typedef enum { FGR_F32 = 0, FGR_BF16 = 1 } fgr_dtype;
-typedef enum { FGR_ACT_NONE = 0, FGR_ACT_RELU = 1, FGR_ACT_GELU_TANH = 2 } fgr_act;
+typedef enum { FGR_ACT_NONE = 0, FGR_ACT_RELU = 1, FGR_ACT_GELU_TANH = 2, FGR_ACT_SIGMOID = 3, FGR_ACT_TANH = 4,
+               FGR_ACT_SILU = 5 } fgr_act;
 typedef enum { FGR_SCALE_NONE = 0, FGR_SCALE_SCALAR = 1, FGR_SCALE_PER_COLUMN = 2 } fgr_scale_kind;
 typedef enum { FGR_RED_LSE = 0, FGR_RED_SOFTMAX = 1, FGR_RED_MAXSUM = 2, FGR_RED_MAX_SUMEXP = 3 } fgr_reduce;
 

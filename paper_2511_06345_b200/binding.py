@@ -14,7 +14,7 @@ LIB_PATH = os.path.join(_HERE, "libfgr.so")
 FGR_OK, FGR_ERR_INVALID_ARG, FGR_ERR_UNSUPPORTED, FGR_ERR_WORKSPACE = 0, 1, 2, 3
 FGR_ERR_CUDA, FGR_ERR_DEVICE_TIMEOUT, FGR_ERR_ARCH = 4, 5, 6
 FGR_F32, FGR_BF16 = 0, 1
-FGR_ACT_NONE, FGR_ACT_RELU, FGR_ACT_GELU_TANH = 0, 1, 2
+FGR_ACT_NONE, FGR_ACT_RELU, FGR_ACT_GELU_TANH, FGR_ACT_SIGMOID, FGR_ACT_TANH, FGR_ACT_SILU = 0, 1, 2, 3, 4, 5
 FGR_SCALE_NONE, FGR_SCALE_SCALAR, FGR_SCALE_PER_COLUMN = 0, 1, 2
 FGR_RED_LSE, FGR_RED_SOFTMAX, FGR_RED_MAXSUM, FGR_RED_MAX_SUMEXP = 0, 1, 2, 3
 FGR_REDUCE_MAX, FGR_REDUCE_SUM = 4, 5

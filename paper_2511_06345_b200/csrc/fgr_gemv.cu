@@ -24,6 +24,9 @@ __device__ __forceinline__ float activation(int act, float u) {
     const float c = 0.7978845608028654f;  // sqrt(2 / pi)
     return 0.5f * u * (1.0f + tanhf(c * (u + 0.044715f * u * u * u)));
   }
+  if (act == FGR_ACT_SIGMOID) return 1.0f / (1.0f + expf(-u));
+  if (act == FGR_ACT_TANH) return tanhf(u);
+  if (act == FGR_ACT_SILU) return u / (1.0f + expf(-u));
   return u;
 }
 

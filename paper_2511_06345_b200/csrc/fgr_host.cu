@@ -63,7 +63,7 @@ int validate(const fgr_desc* d) {
   if (!d) return FGR_ERR_INVALID_ARG;
   if (d->struct_bytes != sizeof(fgr_desc)) return FGR_ERR_INVALID_ARG;
   if (d->dtype != FGR_F32 && d->dtype != FGR_BF16) return FGR_ERR_INVALID_ARG;
-  if (d->act < FGR_ACT_NONE || d->act > FGR_ACT_GELU_TANH) return FGR_ERR_INVALID_ARG;
+  if (d->act < FGR_ACT_NONE || d->act > FGR_ACT_SILU) return FGR_ERR_INVALID_ARG;
   if (d->scale_kind < FGR_SCALE_NONE || d->scale_kind > FGR_SCALE_PER_COLUMN) return FGR_ERR_INVALID_ARG;
   if (d->reduce < FGR_RED_LSE || d->reduce > FGR_RED_MAX_SUMEXP) return FGR_ERR_INVALID_ARG;
   if (d->force_path < FGR_PATH_AUTO || d->force_path > FGR_PATH_SIMT_GEMV) return FGR_ERR_INVALID_ARG;

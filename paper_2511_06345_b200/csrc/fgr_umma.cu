@@ -8,6 +8,9 @@ cudaError_t umma_prepare(int) {
   cudaError_t e = umma_prepare_act_none();
   if (e == cudaSuccess) e = umma_prepare_act_relu();
   if (e == cudaSuccess) e = umma_prepare_act_gelu();
+  if (e == cudaSuccess) e = umma_prepare_act_sigmoid();
+  if (e == cudaSuccess) e = umma_prepare_act_tanh();
+  if (e == cudaSuccess) e = umma_prepare_act_silu();
   return e;
 }
 
@@ -22,6 +25,9 @@ cudaError_t launch_umma(const Params& p, const void* tmap_x, const void* tmap_w,
     case FGR_ACT_NONE: return umma_launch_act_none(sc, p.reduce, wy, p, tmap_x, tmap_w, grid, smem_bytes, stream);
     case FGR_ACT_RELU: return umma_launch_act_relu(sc, p.reduce, wy, p, tmap_x, tmap_w, grid, smem_bytes, stream);
     case FGR_ACT_GELU_TANH: return umma_launch_act_gelu(sc, p.reduce, wy, p, tmap_x, tmap_w, grid, smem_bytes, stream);
+    case FGR_ACT_SIGMOID: return umma_launch_act_sigmoid(sc, p.reduce, wy, p, tmap_x, tmap_w, grid, smem_bytes, stream);
+    case FGR_ACT_TANH: return umma_launch_act_tanh(sc, p.reduce, wy, p, tmap_x, tmap_w, grid, smem_bytes, stream);
+    case FGR_ACT_SILU: return umma_launch_act_silu(sc, p.reduce, wy, p, tmap_x, tmap_w, grid, smem_bytes, stream);
     default: return cudaErrorInvalidValue;
   }
 }

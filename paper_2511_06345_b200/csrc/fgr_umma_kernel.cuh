@@ -205,6 +205,13 @@ __device__ __forceinline__ float activation(float u) {
     constexpr float k = -2.0f * 0.7978845608028654f * 1.4426950408889634f;   // -2 sqrt(2/pi) log2(e)
     const float w = fmaf(k * 0.044715f, u * u, k);
     return __fdividef(u, 1.0f + ex2(u * w));
+  } else if constexpr (ACT == FGR_ACT_SIGMOID) {
+    return __fdividef(1.0f, 1.0f + ex2(-1.4426950408889634f * u));
+  } else if constexpr (ACT == FGR_ACT_TANH) {
+    // tanh u = 1 - 2 / (1 + e^(2u)); for large u the quotient underflows to 0, for very negative u it is 2
+    return 1.0f - __fdividef(2.0f, 1.0f + ex2(2.0f * 1.4426950408889634f * u));
+  } else if constexpr (ACT == FGR_ACT_SILU) {
+    return __fdividef(u, 1.0f + ex2(-1.4426950408889634f * u));
   } else {
     return u;
   }
@@ -606,6 +613,12 @@ cudaError_t prepare_act() {
 cudaError_t umma_launch_act_none(bool sc, int red, bool wy, const Params& p, const void* tx, const void* tw, int grid, int smem, cudaStream_t s);
 cudaError_t umma_launch_act_relu(bool sc, int red, bool wy, const Params& p, const void* tx, const void* tw, int grid, int smem, cudaStream_t s);
 cudaError_t umma_launch_act_gelu(bool sc, int red, bool wy, const Params& p, const void* tx, const void* tw, int grid, int smem, cudaStream_t s);
+cudaError_t umma_launch_act_sigmoid(bool sc, int red, bool wy, const Params& p, const void* tx, const void* tw, int grid, int smem, cudaStream_t s);
+cudaError_t umma_prepare_act_sigmoid();
+cudaError_t umma_launch_act_tanh(bool sc, int red, bool wy, const Params& p, const void* tx, const void* tw, int grid, int smem, cudaStream_t s);
+cudaError_t umma_prepare_act_tanh();
+cudaError_t umma_launch_act_silu(bool sc, int red, bool wy, const Params& p, const void* tx, const void* tw, int grid, int smem, cudaStream_t s);
+cudaError_t umma_prepare_act_silu();
 cudaError_t umma_prepare_act_none();
 cudaError_t umma_prepare_act_relu();
 cudaError_t umma_prepare_act_gelu();

@@ -89,7 +89,7 @@ def test_forced_tiles_and_paths():
     (dict(N=12), fgr.FGR_ERR_UNSUPPORTED),            # bf16 needs N % 8 == 0
     (dict(K=20), fgr.FGR_ERR_UNSUPPORTED),
     (dict(M=0), fgr.FGR_ERR_INVALID_ARG),
-    (dict(act=3), fgr.FGR_ERR_INVALID_ARG),
+    (dict(act=6), fgr.FGR_ERR_INVALID_ARG),
     (dict(reduce=4), fgr.FGR_ERR_INVALID_ARG),
     (dict(dtype=2), fgr.FGR_ERR_INVALID_ARG),
     (dict(ldx=8), fgr.FGR_ERR_INVALID_ARG),           # smaller than K

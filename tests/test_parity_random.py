@@ -31,7 +31,7 @@ def _draw(rng):
             kw["force_cta_pair"] = int(rng.choice([0, 1, 2]))
             if kw["force_cta_pair"] == 2 and kw["force_tile_n"] == 0 and N < 256 and ((N + 15) // 16 * 16) % 32:
                 kw["force_cta_pair"] = 0          # the automatic width would not halve into whole 16-row groups
-    p = gi.make_problem("rnd", B, M, N, K, dtype, int(rng.integers(0, 3)), int(rng.integers(0, 3)), red,
+    p = gi.make_problem("rnd", B, M, N, K, dtype, int(rng.integers(0, 6)), int(rng.integers(0, 3)), red,
                         scale=float(rng.choice([0.5, -1.25, 3.0])), write_y=int(rng.integers(0, 2)), x_std=1.0,
                         w_std=2.0 / np.sqrt(K), bias_range=(-0.5, 0.5) if rng.random() < 0.8 else None,
                         scale_range=(-1.5, 1.5), bias_per_batch=int(rng.integers(0, 2)), seed=int(rng.integers(1, 1 << 30)))

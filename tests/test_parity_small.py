@@ -10,7 +10,7 @@ from parity import compare, run_gpu, to_device
 
 pytestmark = pytest.mark.gpu
 
-ACTS = [gi.ACT_NONE, gi.ACT_RELU, gi.ACT_GELU_TANH]
+ACTS = [gi.ACT_NONE, gi.ACT_RELU, gi.ACT_GELU_TANH, gi.ACT_SIGMOID, gi.ACT_TANH, gi.ACT_SILU]
 REDS = [gi.RED_LSE, gi.RED_SOFTMAX, gi.RED_MAXSUM, gi.RED_MAX_SUMEXP]
 
 
