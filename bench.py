@@ -28,7 +28,19 @@ sys.path.insert(0, ROOT)
 L2_BYTES = 126e6
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 METRIC = "fused GEMM+epilogue+rowreduce TFLOP/s (or GB/s) and % of roofline, 1 B200"
-HBM_BOUND = {"c4"}
+HBM_BOUND = {"c4", "g2"}
+# extra workloads of the fused operator beside the five named ones: the skinny CUDA-core GEMV path
+EXTRA_CONFIGS = {"g2": ("c4", dict(M=2))}     # c4's shapes and epilogue with M = 2
+
+
+def make_cfg(name, **kw):
+    import fgr_inputs as gi
+    if name in EXTRA_CONFIGS:
+        base, over = EXTRA_CONFIGS[name]
+        p = gi.make_config(base, **dict(over, **kw))
+        p.name = name
+        return p
+    return gi.make_config(name, **kw)
 
 
 def load_peaks():
@@ -154,7 +166,7 @@ def run_reference(args):
     if rank != 0:
         return
     import fgr_inputs as gi
-    p = gi.make_config(args.config, seed=0)
+    p = make_cfg(args.config, seed=0)
     per_step = min(2.0, 60.0 / max(args.steps, 1))   # the whole run stays near a minute of CPU time
     flop = dt = 0.0
     threads = rows = 0
@@ -199,7 +211,7 @@ def run_ours(args):
 
     sampler = ClockSampler(local_rank)
     # ---- inputs: a rotation of distinct problems so that no step finds its operands in L2
-    shape = gi.make_config(cfg, materialize=False)
+    shape = make_cfg(cfg, materialize=False)
     set_bytes = shape.min_bytes()
     rot = max(2, int(math.ceil(2.4 * L2_BYTES / set_bytes)) + 1)
     rot = min(rot, 8)
@@ -215,7 +227,7 @@ def run_ours(args):
     sets = []
     host0 = None
     for r, seed in enumerate(rank_seeds(rank, rot)):
-        p = gi.make_config(cfg, seed=seed)
+        p = make_cfg(cfg, seed=seed)
         if r == 0:
             host0 = p
         sets.append(dict(X=up(p.X, b16), W=up(p.W, b16),
@@ -287,7 +299,8 @@ def run_ours(args):
                 "frac_of_sustained_peak": p.flop / kern_s / 1e12 / peaks["bf16_tflops_sustained"]}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["peak_source"] = peak_src + (" (burst)" if roof["bound"] == "tensor" else "")
-    roof["kernel"] = "umma_kernel" if plan.path in (fgr.FGR_PATH_UMMA_TILED, fgr.FGR_PATH_UMMA_STREAM_W) else "simt_gemm_kernel"
+    roof["kernel"] = {fgr.FGR_PATH_UMMA_TILED: "umma_kernel", fgr.FGR_PATH_UMMA_STREAM_W: "umma_kernel",
+                      fgr.FGR_PATH_SIMT_GEMV: "gemv_kernel"}.get(plan.path, "simt_gemm_kernel")
     roof["kernel_us"] = kern_s * 1e6
     roof["timing"] = "CUDA events around each of %d launches of the kernel, in a second pass of the same steps" % kern_runs
     roof["traffic"] = TRAFFIC.get(cfg)
@@ -429,7 +442,8 @@ def run_reduce(args):
                 "clocks": sampler.summary(t0, t1), "gpu_launches": args.steps,
                 "roofline": {"bound": "hbm", "achieved": value / world, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                              "frac": value / world / peaks["hbm_gbs"], "peak_source": peak_src, "kernel": "reduce_rows_kernel",
-                             "kernel_us": ms_step * 1e3, "timing": "the step is this one kernel", "traffic": None},
+                             "kernel_us": ms_step * 1e3, "timing": "the step is this one kernel",
+                             "traffic": TRAFFIC.get(args.config)},
                 "e2e": {"value": world * nbytes / dt / 1e9, "unit": "GB/s", "h2d_bytes_per_step": M * N * 2,
                         "d2h_bytes_per_step": res_h.numel() * res_h.element_size(), "steps": e2e_steps, "ms_per_step": dt * 1e3}}
         if cpu:
@@ -442,7 +456,8 @@ def run_reduce(args):
 # DRAM bytes per launch of the main kernel from ncu (dram__bytes_read.sum + dram__bytes_write.sum), one
 # capture per workload of the kernel as it stands (profiles/umma_kernel_<workload>.md); a workload
 # without a capture of the current kernel reports null.
-TRAFFIC = {"c2": 84.17e6, "c3": 171.70e6, "c4": 274.74e6, "c5": 70.83e6}
+TRAFFIC = {"c2": 84.17e6, "c3": 171.70e6, "c4": 274.74e6, "c5": 70.83e6, "g2": 272.65e6,
+           "r_max": 138.37e6, "r_lse": 138.14e6, "r_softmax": 225.07e6}
 
 
 def main():
@@ -451,7 +466,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5"] + sorted(REDUCE_CONFIGS))
+    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5"] + sorted(EXTRA_CONFIGS) + sorted(REDUCE_CONFIGS))
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
