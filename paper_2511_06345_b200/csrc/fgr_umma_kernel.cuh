@@ -221,13 +221,25 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&r);
 }
 
-// 16 fp32 -> 16 bf16 to global memory; the first 8 (16 bytes) always, the second 8 if `both`.
+// 16 fp32 -> 16 bf16 to global memory; the first 8 (16 bytes) always, the second 8 if `both`.  A
+// 32-byte aligned pair goes out as one 256-bit store: a whole 32-byte sector per lane, which the L2
+// takes as one full-sector write instead of two partial ones.
 __device__ __forceinline__ void store_bf16x16(__nv_bfloat16* dst, const float* y, bool both) {
-  *reinterpret_cast<uint4*>(dst) =
-      make_uint4(pack_bf16(y[0], y[1]), pack_bf16(y[2], y[3]), pack_bf16(y[4], y[5]), pack_bf16(y[6], y[7]));
-  if (both)
-    *reinterpret_cast<uint4*>(dst + 8) =
-        make_uint4(pack_bf16(y[8], y[9]), pack_bf16(y[10], y[11]), pack_bf16(y[12], y[13]), pack_bf16(y[14], y[15]));
+  const uint32_t w0 = pack_bf16(y[0], y[1]), w1 = pack_bf16(y[2], y[3]), w2 = pack_bf16(y[4], y[5]), w3 = pack_bf16(y[6], y[7]);
+  if (both) {
+    const uint32_t w4 = pack_bf16(y[8], y[9]), w5 = pack_bf16(y[10], y[11]), w6 = pack_bf16(y[12], y[13]),
+                   w7 = pack_bf16(y[14], y[15]);
+    if ((reinterpret_cast<uintptr_t>(dst) & 31u) == 0) {
+      asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(w0), "r"(w1), "r"(w2), "r"(w3),
+                   "r"(w4), "r"(w5), "r"(w6), "r"(w7)
+                   : "memory");
+    } else {
+      *reinterpret_cast<uint4*>(dst) = make_uint4(w0, w1, w2, w3);
+      *reinterpret_cast<uint4*>(dst + 8) = make_uint4(w4, w5, w6, w7);
+    }
+  } else {
+    *reinterpret_cast<uint4*>(dst) = make_uint4(w0, w1, w2, w3);
+  }
 }
 
 // Work unit t -> (batch, first row of this CTA, first column).  A unit is one 128-row tile, or for
