@@ -227,7 +227,9 @@ __global__ void __launch_bounds__(256) normalise_kernel(const Params p) {
   extern __shared__ float factor[];   // [parts_per_row]
   let_next_kernel_start();
   wait_for_prior_kernel();
-  const long long row = blockIdx.x;
+  // The GEMM pass writes rows in ascending order, so the rows written last are the ones still in L2:
+  // take them first, before this pass's own traffic evicts them.
+  const long long row = (long long)gridDim.x - 1 - blockIdx.x;
   const int bt = (int)(row / p.M), m = (int)(row % p.M);
   const float2* src = reinterpret_cast<const float2*>(p.parts) + row * p.parts_per_row;
   if (threadIdx.x < 32) {
@@ -270,6 +272,28 @@ __global__ void __launch_bounds__(256) normalise_kernel(const Params p) {
     }
     return raw;
   };
+  if constexpr (sizeof(T) == 2) {
+    // bf16 rows that start on a 32-byte boundary: 256-bit accesses (16 elements, still inside one slot)
+    if ((reinterpret_cast<uintptr_t>(y) & 31u) == 0 && p.N % 16 == 0) {
+      for (int c = threadIdx.x * 16; c < p.N; c += blockDim.x * 16) {
+        uint32_t w[8];
+        asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                     : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+                     : "l"(y + c)
+                     : "memory");
+        const float f = factor[part_slot(c, p.tile_n, p.half_n, p.slots_per_tile)];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          __nv_bfloat162 r = __floats2bfloat162_rn(__uint_as_float(w[j] << 16) * f, __uint_as_float(w[j] & 0xffff0000u) * f);
+          w[j] = *reinterpret_cast<uint32_t*>(&r);
+        }
+        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(y + c), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+                     "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                     : "memory");
+      }
+      return;
+    }
+  }
   const int stride = blockDim.x * V;
   int c = threadIdx.x * V;
   for (; c + stride < p.N; c += 2 * stride) {   // two independent 16-byte accesses in flight per thread
