@@ -453,6 +453,109 @@ def run_reduce(args):
         dist.destroy_process_group()
 
 
+NSHARD_CONFIGS = {"c4n": "c4"}   # the skinny workload with W's rows (N) sharded over the ranks: strong scaling
+
+
+def run_nshard(args):
+    """Bench leg of the N-sharded operator: every rank streams its slice of W, one all-gather of the
+    per-row statistics (rows x 8 bytes per rank, NCCL), then fgr_combine_shards.  The problem is fixed
+    as ranks are added (strong scaling); value = the whole problem's algorithmic bytes / step time."""
+    import numpy as np
+    import torch
+    import fgr_inputs as gi
+    import paper_2511_06345_b200 as fgr
+    rank, local_rank, world = dist_env()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    base = NSHARD_CONFIGS[args.config]
+    peaks, peak_src = load_peaks()
+    shape = make_cfg(base, materialize=False)
+    op = fgr.NShardedFusedGemmReduce(shape.batch, shape.M, shape.N, shape.K, shape.dtype, shape.act, shape.scale_kind,
+                                     shape.reduce, scale=shape.scale, device=local_rank)
+    n0, n1 = op.n0, op.n1
+    slice_bytes = (n1 - n0) * shape.K * 2 + shape.M * shape.K * 2
+    rot = min(8, max(2, int(math.ceil(2.4 * L2_BYTES / slice_bytes)) + 1))
+    up16 = lambda a: torch.from_numpy(np.ascontiguousarray(a)).view(torch.int16).view(torch.bfloat16).to(dev)
+    sets, host0 = [], None
+    for seed in range(rot):                       # all ranks draw the same problems and keep their slice
+        p = make_cfg(base, seed=seed)
+        sets.append((up16(p.X), up16(p.W[:, n0:n1, :]), torch.from_numpy(p.bias[n0:n1].copy()).to(dev)))
+        host0 = host0 or p
+    p = host0
+    step = lambda i: op(*sets[i % rot])
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    e0.record()
+    for i in range(args.steps):
+        _, out = step(i)
+    e1.record()
+    barrier()
+    t1 = time.perf_counter()
+    if op.status() != fgr.FGR_OK:
+        raise SystemExit("device status after the timed region: " + fgr.fgr_status_string(op.status()))
+    ms_step = max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps
+    h = op.local.handle
+    fgr.fgr_profile_enable(h, True)
+    for i in range(args.steps):
+        step(i)
+    barrier()
+    sampler.stop()
+    kern_ms, kern_runs = fgr.fgr_profile_read(h)
+    kern_s = kern_ms / max(kern_runs, 1) * 1e-3
+    value = p.min_bytes() / (ms_step * 1e-3) / 1e9
+    local_bytes = slice_bytes + (n1 - n0) * 4 + p.M * 8
+    roof = {"bound": "hbm", "achieved": local_bytes / kern_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "peak_source": peak_src, "kernel": "umma_kernel", "kernel_us": kern_s * 1e6, "traffic": None,
+            "timing": "CUDA events around each of %d launches of the rank-local main kernel (its slice: %d columns)" % (kern_runs, n1 - n0)}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    # end to end: this rank's host slice in, the result out
+    hp = [t.cpu().pin_memory() for t in sets[0]]
+    res = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+    e2e_steps = max(3, min(args.steps, 20))
+
+    def e2e_step():
+        for d, s_ in zip(sets[0], hp):
+            d.copy_(s_, non_blocking=True)
+        res.copy_(op(*sets[0])[1], non_blocking=True)
+        torch.cuda.synchronize(dev)
+    e2e_step()
+    barrier()
+    te = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    dt = max_over_ranks((time.perf_counter() - te) / e2e_steps, world, dev)
+    if rank == 0:
+        plan = op.local.plan
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": args.config, "batch": p.batch, "M": p.M, "N": p.N, "K": p.K, "act": "gelu_tanh",
+                       "reduce": "lse", "path": fgr.fgr_path_name(plan.path), "tile": [plan.tile_m, plan.tile_n],
+                       "columns_per_rank": n1 - n0,
+                       "l2": "rotating %d distinct input sets per rank (%.0f MB > 126 MB L2)" % (rot, rot * slice_bytes / 1e6),
+                       "parallelism": "N sharded over %d rank(s); all-gather of [rows, 2] fp32 + combine kernel" % world},
+            "clocks": sampler.summary(t0, t1), "gpu_launches": args.steps * (plan.launches + 1), "roofline": roof,
+            "e2e": {"value": p.min_bytes() / dt / 1e9, "unit": "GB/s", "h2d_bytes_per_step": sum(t.numel() * t.element_size() for t in hp),
+                    "d2h_bytes_per_step": res.numel() * 4, "steps": e2e_steps, "ms_per_step": dt * 1e3}}))
+    op.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
 # DRAM bytes per launch of the main kernel from ncu (dram__bytes_read.sum + dram__bytes_write.sum), one
 # capture per workload of the kernel as it stands (profiles/umma_kernel_<workload>.md); a workload
 # without a capture of the current kernel reports null.
@@ -466,11 +569,17 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5"] + sorted(EXTRA_CONFIGS) + sorted(REDUCE_CONFIGS))
+    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5"] + sorted(EXTRA_CONFIGS) + sorted(REDUCE_CONFIGS) + sorted(NSHARD_CONFIGS))
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
-    if args.config in REDUCE_CONFIGS:
+    if args.config in NSHARD_CONFIGS:
+        if args.impl == "reference":
+            args.config = NSHARD_CONFIGS[args.config]     # the oracle has no shards: the same workload, whole
+            run_reference(args)
+        else:
+            run_nshard(args)
+    elif args.config in REDUCE_CONFIGS:
         if args.impl == "reference":
             raise SystemExit("the reference arm covers the fused operator's workloads c1..c5")
         run_reduce(args)

@@ -146,7 +146,9 @@ FGR_API int fgr_get_plan(const fgr_handle* h, fgr_plan_info* info /*host, out*/)
  *   bias       device fp32 [N] (or [batch, N]); NULL = no bias
  *   scale_vec  device fp32 [N]; required iff scale_kind == FGR_SCALE_PER_COLUMN
  *   Y          device, dtype, [batch, M, N]; required iff write_y or SOFTMAX
- *   out        device fp32: [batch*M] (LSE) or [batch*M, 2] (MAXSUM, MAX_SUMEXP); NULL for SOFTMAX
+ *   out        device fp32: [batch*M] (LSE) or [batch*M, 2] (MAXSUM, MAX_SUMEXP).  SOFTMAX: optional;
+ *              if not NULL it receives [batch*M, 2] = (row max, sum of exp(y - max)), the statistics
+ *              that P was normalised with (what fgr_combine_shards needs)
  *   workspace  device, 256-byte aligned, at least fgr_workspace_bytes(h); scratch for the
  *              split-N partial pairs and the device status word.  Two runs that overlap in time
  *              must not share a workspace.
@@ -227,6 +229,41 @@ typedef struct fgr_reduce_desc {
   int64_t lda, ldp;        /* row strides in elements; 0 = packed */
 } fgr_reduce_desc;
 FGR_API int fgr_reduce_rows(const fgr_reduce_desc* desc /*host*/, const void* A, void* P, float* out, void* cuda_stream);
+
+/*
+ * fgr_combine_shards: the exchange step's local half when N is sharded over several GPUs (one
+ * process per GPU).  The operator's rows are independent, so sharding over rows or batches needs no
+ * exchange; sharding over N (the sensible split for a skinny, weight-streaming problem, where W is
+ * almost all of the bytes) leaves every GPU with the statistics of its own column slice.  The
+ * problem statement is unchanged: the same outputs as the unsharded operator (Section 3.1,
+ * Verifier; Section 3.3).  Protocol, per GPU g of G:
+ *   1. fgr_run on the slice W[n_g0:n_g1, :] (bias and scale slices alike) with reduce =
+ *      FGR_RED_MAX_SUMEXP (for a final LSE or MAX_SUMEXP), FGR_RED_MAXSUM (final MAXSUM) or
+ *      FGR_RED_SOFTMAX with `out` given (final softmax) -> a local pair per row, [rows, 2] fp32;
+ *   2. all-gather of the pairs (NCCL; rows * 8 bytes per GPU) -> pairs[G][rows][2] on every GPU;
+ *   3. fgr_combine_shards merges the G pairs of every row in ascending shard order (so every GPU
+ *      computes bit-identical results) and writes `out` as the unsharded operator would; for softmax
+ *      it rescales the local slice P_local[rows, n_local] in place by l_g exp(m_g - m) / l.
+ *   pairs    device fp32 [shards][rows][2], 8-byte aligned
+ *   out      device fp32 [rows] (LSE) or [rows, 2]; required unless SOFTMAX (there optional: (m, l))
+ *   P_local  device, dtype, row stride ldp (0 = n_local), 16-byte aligned; SOFTMAX only
+ * n_local and ldp must be multiples of 8 (bf16) / 4 (fp32).  One launch on `cuda_stream`,
+ * asynchronous, no workspace.
+ */
+typedef struct fgr_shard_desc {
+  uint32_t struct_bytes;   /* = sizeof(fgr_shard_desc) */
+  int32_t shards;          /* G >= 1 */
+  int32_t reduce;          /* fgr_reduce of the whole operator */
+  int32_t dtype;           /* fgr_dtype of P_local (SOFTMAX only) */
+  int32_t shard;           /* this GPU's index in [0, G) (SOFTMAX only) */
+  int32_t n_local;         /* columns of this GPU's slice (SOFTMAX only) */
+  int32_t device;          /* CUDA device ordinal */
+  int32_t reserved;        /* 0 */
+  int64_t rows;            /* batch * M */
+  int64_t ldp;             /* row stride of P_local in elements; 0 = n_local */
+} fgr_shard_desc;
+FGR_API int fgr_combine_shards(const fgr_shard_desc* desc /*host*/, const float* pairs, float* out, void* P_local,
+                               void* cuda_stream);
 
 /*
  * Timing of the main kernel (the GEMM + epilogue + per-tile reduction launch), for benchmarks.

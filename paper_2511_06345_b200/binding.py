@@ -22,7 +22,7 @@ FGR_PATH_AUTO, FGR_PATH_SIMT, FGR_PATH_UMMA_TILED, FGR_PATH_UMMA_STREAM_W, FGR_P
 
 FGR_STATIC_SCRATCH_BYTES = 4 << 20
 
-EXPORTS = ("fgr_plan", "fgr_create", "fgr_workspace_bytes", "fgr_get_plan", "fgr_run", "fgr_run_host", "fgr_run_static", "fgr_reduce_rows",
+EXPORTS = ("fgr_plan", "fgr_create", "fgr_workspace_bytes", "fgr_get_plan", "fgr_run", "fgr_run_host", "fgr_run_static", "fgr_reduce_rows", "fgr_combine_shards",
            "fgr_get_status", "fgr_profile_enable", "fgr_profile_read", "fgr_destroy", "fgr_status_string", "fgr_path_name")
 
 
@@ -42,6 +42,13 @@ class fgr_reduce_desc(ctypes.Structure):
     _fields_ = [("struct_bytes", ctypes.c_uint32), ("M", ctypes.c_int32), ("N", ctypes.c_int32),
                 ("dtype", ctypes.c_int32), ("reduce", ctypes.c_int32), ("device", ctypes.c_int32),
                 ("lda", ctypes.c_int64), ("ldp", ctypes.c_int64)]
+
+
+class fgr_shard_desc(ctypes.Structure):
+    _fields_ = [("struct_bytes", ctypes.c_uint32), ("shards", ctypes.c_int32), ("reduce", ctypes.c_int32),
+                ("dtype", ctypes.c_int32), ("shard", ctypes.c_int32), ("n_local", ctypes.c_int32),
+                ("device", ctypes.c_int32), ("reserved", ctypes.c_int32), ("rows", ctypes.c_int64),
+                ("ldp", ctypes.c_int64)]
 
 
 class fgr_plan_info(ctypes.Structure):
@@ -81,6 +88,7 @@ def lib() -> ctypes.CDLL:
         L.fgr_run_host.argtypes, L.fgr_run_host.restype = [vp] * 7, i
         L.fgr_run_static.argtypes, L.fgr_run_static.restype = [ctypes.POINTER(fgr_desc)] + [vp] * 7, i
         L.fgr_reduce_rows.argtypes, L.fgr_reduce_rows.restype = [ctypes.POINTER(fgr_reduce_desc)] + [vp] * 4, i
+        L.fgr_combine_shards.argtypes, L.fgr_combine_shards.restype = [ctypes.POINTER(fgr_shard_desc)] + [vp] * 4, i
         L.fgr_get_status.argtypes, L.fgr_get_status.restype = [vp], i
         L.fgr_profile_enable.argtypes, L.fgr_profile_enable.restype = [vp, i], i
         L.fgr_profile_read.argtypes, L.fgr_profile_read.restype = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i)], i
@@ -176,6 +184,17 @@ def fgr_reduce_rows(M, N, dtype, reduce, A, P, out, *, lda=0, ldp=0, device=0, s
     rc = lib().fgr_reduce_rows(ctypes.byref(d), _addr(A), _addr(P), _addr(out), stream)
     if check and rc != FGR_OK:
         raise FgrError(rc, "fgr_reduce_rows")
+    return rc
+
+
+def fgr_combine_shards(rows, shards, reduce, pairs, out, P_local=None, *, dtype=FGR_BF16, shard=0, n_local=0, ldp=0,
+                       device=0, stream=None, check=True) -> int:
+    """Merges the all-gathered per-shard row statistics ``pairs`` [shards, rows, 2] of an N-sharded
+    operator (device pointers: ints or tensors); softmax also rescales the local slice ``P_local``."""
+    d = fgr_shard_desc(ctypes.sizeof(fgr_shard_desc), shards, reduce, dtype, shard, n_local, device, 0, rows, ldp)
+    rc = lib().fgr_combine_shards(ctypes.byref(d), _addr(pairs), _addr(out), _addr(P_local), stream)
+    if check and rc != FGR_OK:
+        raise FgrError(rc, "fgr_combine_shards")
     return rc
 
 

@@ -252,6 +252,8 @@ __global__ void __launch_bounds__(256) normalise_kernel(const Params p) {
     }
     const float inv = 1.0f / l;
     for (int t = lane; t < p.parts_per_row; t += 32) factor[t] *= inv;
+    // optional row statistics (row max, sum of exp(y - max)): what a combine over column shards needs
+    if (lane == 0 && p.out) reinterpret_cast<float2*>(p.out)[row] = make_float2(a, l);
   }
   __syncthreads();
   T* y = static_cast<T*>(p.Y) + (long long)bt * p.bsy + (long long)m * p.ldy;

@@ -56,9 +56,10 @@ def run_gpu(p: gi.Problem, force_path=0, force_tile_n=0, device=0, tensors=None,
     return Yh, oh, plan
 
 
-def compare(p: gi.Problem, Y, out, rows=None, tcgen05=True):
+def compare(p: gi.Problem, Y, out, rows=None, tcgen05=True, softmax_rel=9e-3):
     """Asserts GPU results (all rows, or the listed global rows) against the oracle.  Returns the
-    achieved maxima of |err| / (1 + |ref|) for Y and out."""
+    achieved maxima of |err| / (1 + |ref|) for Y and out.  ``softmax_rel``: relative bound on a bf16 P
+    (4.5e-3 per rounding: two on the single-GPU path, three when a shard combine rescales once more)."""
     Yr, outr, _ = oracle.run_problem(p, rows=rows, want_y=True)
     if rows is not None:
         Y = None if Y is None else Y[rows]
@@ -73,7 +74,7 @@ def compare(p: gi.Problem, Y, out, rows=None, tcgen05=True):
         if p.dtype == gi.DTYPE_F32:
             bound = 1e-5 * np.abs(Yr) + 1e-6 * (1 + big)
         elif p.reduce == gi.RED_SOFTMAX:
-            bound = 9e-3 * np.abs(Yr) + 1e-7
+            bound = softmax_rel * np.abs(Yr) + 1e-7
         else:
             bound = 4.5e-3 * np.abs(Yr) + 2e-5 * (1 + big)
         bad = err > bound
