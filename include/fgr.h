@@ -72,8 +72,11 @@ typedef enum {
   FGR_PATH_SIMT = 1,          /* CUDA-core tiles, fp32 FMA: the fp32 path, also valid for bf16 */
   FGR_PATH_UMMA_TILED = 2,    /* tcgen05 128 x 256 tiles, TMA ring, compute-bound shapes (bf16) */
   FGR_PATH_UMMA_STREAM_W = 3, /* tcgen05 with narrow N tiles and a deep TMA ring: M <= 128, W streamed once (bf16) */
-  FGR_PATH_SIMT_GEMV = 4      /* M <= 16: warps stream rows of W with 128-bit loads, shuffle reductions (bf16; no softmax;
+  FGR_PATH_SIMT_GEMV = 4,     /* M <= 16: warps stream rows of W with 128-bit loads, shuffle reductions (bf16; no softmax;
                                  chosen automatically for M <= 4) */
+  FGR_PATH_UMMA_TF32X3 = 5    /* fp32 on tensor cores: X and W are split into tf32 hi + lo planes (in the workspace) and
+                                 tcgen05 kind::tf32 accumulates hi*hi + hi*lo + lo*hi in fp32; fp32-level accuracy
+                                 (about 2^-21 per product); chosen automatically for large compute-bound fp32 problems */
 } fgr_path;
 
 typedef struct fgr_desc {

@@ -11,7 +11,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(HERE, "libfgr.so")
 SOURCES = ["fgr_host.cu", "fgr_simt.cu", "fgr_umma.cu", "fgr_umma_act_none.cu", "fgr_umma_act_relu.cu",
-           "fgr_umma_act_gelu.cu", "fgr_umma_act_sigmoid.cu", "fgr_umma_act_tanh.cu", "fgr_umma_act_silu.cu", "fgr_gemv.cu", "fgr_reduce.cu", "fgr_noalloc.cu", "fgr_shard.cu"]
+           "fgr_umma_act_gelu.cu", "fgr_umma_act_sigmoid.cu", "fgr_umma_act_tanh.cu", "fgr_umma_act_silu.cu", "fgr_gemv.cu", "fgr_reduce.cu", "fgr_noalloc.cu", "fgr_shard.cu", "fgr_split.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr"]
 

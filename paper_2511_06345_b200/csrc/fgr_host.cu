@@ -42,6 +42,12 @@ namespace {
 // B200 (about 1640 TFLOP/s over about 6.5 TB/s), in flop per byte.
 constexpr double kRidgeFlopPerByte = 250.0;
 constexpr int kDefaultSms = 148;
+// 3xTF32: K elements accumulated inside the tensor core per chunk = 32 * kTf32ChunkBlocks.  The tensor
+// core truncates its fp32 accumulator once per instruction (measured: a relative bias of about 7e-9 per
+// unit of K, towards zero); 128 keeps that below 1e-6, the level of an fp32 FMA loop at K of a few thousand.
+constexpr int kTf32ChunkBlocks = 4;
+constexpr double kTf32MinFlop = 4.0e9;   // below this the fp32 problem stays on the CUDA-core path
+size_t align256(size_t x) { return (x + 255u) & ~(size_t)255u; }
 
 int elem_bytes(int dtype) { return dtype == FGR_F32 ? 4 : 2; }
 int out_width(int reduce) { return reduce == FGR_RED_LSE ? 1 : reduce == FGR_RED_SOFTMAX ? 0 : 2; }
@@ -66,7 +72,7 @@ int validate(const fgr_desc* d) {
   if (d->act < FGR_ACT_NONE || d->act > FGR_ACT_SILU) return FGR_ERR_INVALID_ARG;
   if (d->scale_kind < FGR_SCALE_NONE || d->scale_kind > FGR_SCALE_PER_COLUMN) return FGR_ERR_INVALID_ARG;
   if (d->reduce < FGR_RED_LSE || d->reduce > FGR_RED_MAX_SUMEXP) return FGR_ERR_INVALID_ARG;
-  if (d->force_path < FGR_PATH_AUTO || d->force_path > FGR_PATH_SIMT_GEMV) return FGR_ERR_INVALID_ARG;
+  if (d->force_path < FGR_PATH_AUTO || d->force_path > FGR_PATH_UMMA_TF32X3) return FGR_ERR_INVALID_ARG;
   if (d->batch < 1 || d->M < 1 || d->N < 1 || d->K < 1) return FGR_ERR_INVALID_ARG;
   if (d->write_y != 0 && d->write_y != 1) return FGR_ERR_INVALID_ARG;
   if (d->bias_per_batch != 0 && d->bias_per_batch != 1) return FGR_ERR_INVALID_ARG;
@@ -124,13 +130,17 @@ int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
 
   int path = d.force_path;
   if (path == FGR_PATH_AUTO) {
-    if (d.dtype == FGR_F32) path = FGR_PATH_SIMT;
+    // fp32: CUDA-core FMA tiles, or for large compute-bound problems three tf32 tensor-core products
+    // (the operand split costs one extra pass over X and W, so small or skinny problems stay on FMA)
+    if (d.dtype == FGR_F32) path = (d.M >= 128 && d.N >= 128 && d.K >= 128 && pi.flop >= kTf32MinFlop) ? FGR_PATH_UMMA_TF32X3 : FGR_PATH_SIMT;
     else if (d.M <= 4 && d.reduce != FGR_RED_SOFTMAX) path = FGR_PATH_SIMT_GEMV;   // a few GEMVs: CUDA cores keep up with HBM
     else if (d.M <= 128 && pi.flop / pi.min_bytes < kRidgeFlopPerByte) path = FGR_PATH_UMMA_STREAM_W;
     else path = FGR_PATH_UMMA_TILED;
   }
   if (path == FGR_PATH_SIMT_GEMV && (d.dtype != FGR_BF16 || d.M > 16 || d.reduce == FGR_RED_SOFTMAX)) return FGR_ERR_UNSUPPORTED;
   if ((path == FGR_PATH_UMMA_TILED || path == FGR_PATH_UMMA_STREAM_W) && d.dtype != FGR_BF16) return FGR_ERR_UNSUPPORTED;
+  if (path == FGR_PATH_UMMA_TF32X3 && d.dtype != FGR_F32) return FGR_ERR_UNSUPPORTED;
+  const bool tf32 = path == FGR_PATH_UMMA_TF32X3;
 
   Params p;
   std::memset(&p, 0, sizeof p);
@@ -175,7 +185,7 @@ int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
     // per SM by a third; they need at least two row blocks and a W tile that halves into whole
     // 16-row groups.
     int pair = d.force_cta_pair;
-    if (!pair) pair = (path == FGR_PATH_UMMA_TILED && row_blocks >= 2 && tn % 32 == 0 && sms >= 2) ? 2 : 1;
+    if (!pair) pair = ((path == FGR_PATH_UMMA_TILED || tf32) && row_blocks >= 2 && tn % 32 == 0 && sms >= 2) ? 2 : 1;
     if (pair == 2 && tn % 32 != 0) return FGR_ERR_UNSUPPORTED;
     p.cta_pair = pair;
     p.tiles_m = (d.M + kUmmaTileM * pair - 1) / (kUmmaTileM * pair);
@@ -188,10 +198,12 @@ int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
     // neighbouring 128-byte lines of the same matrix row back to back, which measurably raises the
     // rate at which operands arrive (L2 and DRAM both work in units larger than one line).  Used
     // when at least three such stages fit in shared memory and K is long enough to fill them.
-    int ksub = d.force_ksub;
+    int ksub = tf32 ? 2 : d.force_ksub;   // 3xTF32: the two sub-blocks of a stage are the hi and lo planes
     if (!ksub) ksub = (d.K > kUmmaBlockK && umma_smem_layout(w_rows, 3, 2).total <= kSmemLimit) ? 2 : 1;
-    while (ksub > 1 && umma_smem_layout(w_rows, 2, ksub).total > kSmemLimit) --ksub;
+    while (!tf32 && ksub > 1 && umma_smem_layout(w_rows, 2, ksub).total > kSmemLimit) --ksub;
     p.ksub = ksub;
+    p.k_plane = tf32 ? (d.K + 31) / 32 * 32 : 0;
+    p.chunk_blocks = kTf32ChunkBlocks;
     int stages = kUmmaMaxStages;
     while (stages > 1 && umma_smem_layout(w_rows, stages, ksub).total > kSmemLimit) --stages;
     p.stages = stages;
@@ -218,8 +230,11 @@ int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
   const bool cuda_cores = path == FGR_PATH_SIMT || path == FGR_PATH_SIMT_GEMV;
   pi.cta_pair = cuda_cores ? 1 : p.cta_pair;
   pi.ksub = cuda_cores ? 0 : p.ksub;
-  pi.launches = 2;   // main kernel + (merge | softmax normalise)
+  pi.launches = tf32 ? 4 : 2;   // (operand split of X and of W +) main kernel + (merge | softmax normalise)
   pi.workspace_bytes = (uint64_t)kStatusBytes + (uint64_t)d.batch * d.M * p.parts_per_row * 8ull;
+  if (tf32)   // the hi / lo planes of X and W follow the partial pairs, each on a 256-byte boundary
+    pi.workspace_bytes = align256(align256((size_t)pi.workspace_bytes) + (size_t)d.batch * d.M * 2 * p.k_plane * 4) +
+                         (uint64_t)d.batch * d.N * 2 * p.k_plane * 4;
   *info = pi;
   if (pp) *pp = p;
   return FGR_OK;
@@ -245,14 +260,17 @@ EncodeTiledFn encode_fn() {
 
 // bf16 [batch, rows, K] with strides (ld, bs) -> 3-D map, box = 64 (K) x box_rows x 1, 128-byte swizzle,
 // out-of-range elements read as zero.
-int encode_operand(CUtensorMap* map, const void* ptr, int K, int rows, int batch, long long ld, long long bs, int box_rows) {
+// (fp32 = true: 4-byte elements, box = 32 (K) x box_rows x 1, the same 128-byte rows.)
+int encode_operand(CUtensorMap* map, const void* ptr, int K, int rows, int batch, long long ld, long long bs, int box_rows,
+                   bool fp32 = false) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return FGR_ERR_CUDA;
+  const unsigned eb = fp32 ? 4 : 2;
   cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)batch};
-  cuuint64_t strides[2] = {(cuuint64_t)ld * 2, (cuuint64_t)(batch > 1 ? bs : (long long)rows * ld) * 2};
-  cuuint32_t box[3] = {(cuuint32_t)kUmmaBlockK, (cuuint32_t)box_rows, 1};
+  cuuint64_t strides[2] = {(cuuint64_t)ld * eb, (cuuint64_t)(batch > 1 ? bs : (long long)rows * ld) * eb};
+  cuuint32_t box[3] = {(cuuint32_t)(kUmmaBlockK * 2 / eb), (cuuint32_t)box_rows, 1};
   cuuint32_t estr[3] = {1, 1, 1};
-  CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+  CUresult rc = fn(map, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return rc == CUDA_SUCCESS ? FGR_OK : FGR_ERR_CUDA;
@@ -292,7 +310,7 @@ int fgr_create(const fgr_desc* desc, fgr_handle** out) {
   h->num_sms = sms;
   rc = make_plan(*desc, sms, &h->plan, &h->base);
   if (rc != FGR_OK) { delete h->events; delete h; return rc; }
-  if (h->plan.path == FGR_PATH_UMMA_TILED || h->plan.path == FGR_PATH_UMMA_STREAM_W) {
+  if (h->plan.path == FGR_PATH_UMMA_TILED || h->plan.path == FGR_PATH_UMMA_STREAM_W || h->plan.path == FGR_PATH_UMMA_TF32X3) {
     int prev = 0;
     cudaGetDevice(&prev);
     cudaError_t e = cudaSetDevice(desc->device);
@@ -357,6 +375,22 @@ int fgr_run(fgr_handle* h, const void* X, const void* W, const float* bias, cons
       e = launch_simt(p, stream);
     } else if (h->plan.path == FGR_PATH_SIMT_GEMV) {
       e = launch_gemv(p, p.tiles_n, p.tile_n, stream);
+    } else if (h->plan.path == FGR_PATH_UMMA_TF32X3) {
+      // split X and W into tf32 hi / lo planes inside the workspace, then the tensor-core kernel on the planes
+      char* wsb = static_cast<char*>(workspace);
+      const size_t x_off = align256((size_t)kStatusBytes + (size_t)d.batch * d.M * p.parts_per_row * 8u);
+      const size_t w_off = align256(x_off + (size_t)d.batch * d.M * 2 * p.k_plane * 4);
+      float* xp = reinterpret_cast<float*>(wsb + x_off);
+      float* wp = reinterpret_cast<float*>(wsb + w_off);
+      e = launch_split_tf32(static_cast<const float*>(X), xp, d.batch, d.M, d.K, p.ldx, p.bsx, p.k_plane, stream);
+      if (e == cudaSuccess) e = launch_split_tf32(static_cast<const float*>(W), wp, d.batch, d.N, d.K, p.ldw, p.bsw, p.k_plane, stream);
+      if (workspace != h->cached_x) {   // the tensor maps describe the planes, which live in the workspace
+        const long long ldp = 2LL * p.k_plane;
+        rc = encode_operand(&h->tmap_x, xp, (int)ldp, d.M, d.batch, ldp, (long long)d.M * ldp, kUmmaTileM, true);
+        if (rc == FGR_OK) rc = encode_operand(&h->tmap_w, wp, (int)ldp, d.N, d.batch, ldp, (long long)d.N * ldp, p.tile_n / p.cta_pair, true);
+        h->cached_x = rc == FGR_OK ? workspace : nullptr;
+      }
+      if (rc == FGR_OK && e == cudaSuccess) e = launch_umma(p, &h->tmap_x, &h->tmap_w, h->plan.grid, h->plan.smem_bytes, stream);
     } else {
       if (X != h->cached_x) {
         rc = encode_operand(&h->tmap_x, X, d.K, d.M, d.batch, p.ldx, p.bsx, kUmmaTileM);
@@ -519,6 +553,7 @@ const char* fgr_path_name(int path) {
     case FGR_PATH_UMMA_TILED: return "umma_tiled";
     case FGR_PATH_UMMA_STREAM_W: return "umma_stream_w";
     case FGR_PATH_SIMT_GEMV: return "simt_gemv";
+    case FGR_PATH_UMMA_TF32X3: return "umma_tf32x3";
     default: return "unknown";
   }
 }

@@ -39,6 +39,8 @@ struct Params {
   int stages;
   int ksub;            // tcgen05 paths: 64-wide K sub-blocks per ring stage (1, 2 or 4)
   int cta_pair;        // tcgen05 paths: 1 = each CTA works alone, 2 = clusters of two CTAs share 256-row tiles
+  int k_plane;         // 3xTF32 path: K rounded up to 32 = width of the hi plane (the lo plane follows it)
+  int chunk_blocks;    // 3xTF32 path: 32-wide k-blocks accumulated in tensor memory before the epilogue adds them up
 };
 
 // Column -> partial-slot mapping shared by the producers of the partials and the normalise pass.
@@ -74,6 +76,10 @@ __host__ __device__ inline UmmaSmem umma_smem_layout(int w_rows, int stages, int
 cudaError_t launch_simt(const Params& p, cudaStream_t stream);
 cudaError_t launch_merge(const Params& p, cudaStream_t stream);
 cudaError_t launch_normalise(const Params& p, cudaStream_t stream);
+// 3xTF32 path: splits fp32 src [batch][rows][K] (strides ld, bs) into dst [batch][rows][2 * k_plane]
+// = [hi | lo], hi = x rounded to tf32, lo = x - hi rounded to tf32, zero beyond K.
+cudaError_t launch_split_tf32(const float* src, float* dst, int batch, int rows, int K, long long ld, long long bs,
+                              int k_plane, cudaStream_t stream);
 cudaError_t launch_gemv(const Params& p, int grid, int rows_per_cta, cudaStream_t stream);
 int gemv_rows_per_warp(int M);
 int gemv_k_chunk(int M, int K);

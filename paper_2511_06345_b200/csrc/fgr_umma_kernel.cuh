@@ -23,6 +23,8 @@
 #include <cuda_bf16.h>
 #include <math_constants.h>
 
+#include <type_traits>
+
 #include "fgr_internal.h"
 
 namespace fgr {
@@ -106,6 +108,16 @@ __device__ __forceinline__ void tcgen05_mma_bf16(uint32_t d_tmem, uint64_t a_des
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// The same with tf32 operands (fp32 words whose low 13 mantissa bits the tensor core ignores), K = 8.
+__device__ __forceinline__ void tcgen05_mma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                 uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 // 32 lanes x 16 consecutive 32-bit columns: thread i of the warp gets lane (base + i), register j =
 // column j.  The load is asynchronous: tcgen05_wait_ld() must precede the first use of r.
 __device__ __forceinline__ void tcgen05_ld16_issue(uint32_t taddr, uint32_t* r) {
@@ -168,6 +180,16 @@ __device__ __forceinline__ void tcgen05_mma_bf16_pair(uint32_t d_tmem, uint64_t 
       : "memory");
 }
 
+__device__ __forceinline__ void tcgen05_mma_tf32_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                      uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
@@ -185,10 +207,11 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
   d |= (uint64_t)2 << 61;                     // 128-byte swizzle
   return d;
 }
-// Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = 128 (256 for a CTA
-// pair), N = tile_n.
-__device__ __forceinline__ uint32_t make_idesc(int tile_m, int tile_n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(tile_n >> 3) << 17) | ((uint32_t)(tile_m >> 4) << 24);
+// Instruction descriptor: D fp32; A and B both bf16 (kind::f16, format code 1) or both tf32
+// (kind::tf32, format code 2), both K-major; M = 128 (256 for a CTA pair), N = tile_n.
+__device__ __forceinline__ uint32_t make_idesc(int tile_m, int tile_n, bool tf32) {
+  const uint32_t fmt = tf32 ? 2u : 1u;
+  return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(tile_n >> 3) << 17) | ((uint32_t)(tile_m >> 4) << 24);
 }
 
 __device__ __forceinline__ float ex2(float x) {
@@ -242,6 +265,13 @@ __device__ __forceinline__ void store_bf16x16(__nv_bfloat16* dst, const float* y
   }
 }
 
+// 16 fp32 to global memory, the first `nv` of them (a multiple of 4) if fewer than 16 are real.
+__device__ __forceinline__ void store_f32x16(float* dst, const float* y, int nv) {
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    if (4 * q < nv) *reinterpret_cast<float4*>(dst + 4 * q) = make_float4(y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]);
+}
+
 // Work unit t -> (batch, first row of this CTA, first column).  A unit is one 128-row tile, or for
 // a CTA pair a 256-row tile of which CTA `rank` owns rows [128 rank, 128 rank + 128).
 struct TileCoord { int bt, m0, n0; };
@@ -288,6 +318,26 @@ __device__ __forceinline__ void apply16(const uint32_t* r, const float* bias_s, 
   }
 }
 
+// the same from 16 fp32 sums held in registers
+template <int ACT, bool SC>
+__device__ __forceinline__ void apply16f(const float* z, const float* bias_s, const float* scale_s, float* y) {
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const float4 b = *reinterpret_cast<const float4*>(bias_s + 4 * q);
+    const float bb[4] = {b.x, b.y, b.z, b.w};
+    float ss[4] = {1.f, 1.f, 1.f, 1.f};
+    if constexpr (SC) {
+      const float4 s = *reinterpret_cast<const float4*>(scale_s + 4 * q);
+      ss[0] = s.x; ss[1] = s.y; ss[2] = s.z; ss[3] = s.w;
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float a = activation<ACT>(z[4 * q + j] + bb[j]);
+      y[4 * q + j] = SC ? a * ss[j] : a;
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------------------ kernel
 // PAIR = false: every CTA works alone on 128 x tile_n tiles (tcgen05 cta_group::1).
 // PAIR = true : the grid is launched in clusters of two CTAs that share 256 x tile_n tiles.  Each
@@ -298,7 +348,12 @@ __device__ __forceinline__ void apply16(const uint32_t* r, const float* bias_s, 
 //   "full" lives in the leader (both CTAs' TMA loads count their bytes there), "empty" and
 //   "tmem_full" are signalled in both CTAs by one multicast tcgen05.commit, "tmem_empty" lives in
 //   the leader and collects the epilogue warps of both CTAs.
-template <int ACT, bool SC, int RED, bool WY, bool PAIR>
+// TF32 = true: fp32 problem computed as three tf32 products (3xTF32).  The operands arrive already
+//   split by split_tf32_kernel into a "hi" plane (x rounded to tf32) and a "lo" plane (x - hi), side
+//   by side along K: [rows][2 * k_plane].  A ring stage holds one 32-wide k-block of all four tiles
+//   (sub-block 0 = X_hi, W_hi; sub-block 1 = X_lo, W_lo) and the MMA warp accumulates
+//   X_hi W_hi + X_hi W_lo + X_lo W_hi into the one fp32 accumulator; Y / P are stored as fp32.
+template <int ACT, bool SC, int RED, bool WY, bool PAIR, bool TF32>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const Params p) {
   using V = Variant<ACT, SC, RED, WY>;
@@ -318,8 +373,13 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L.misc_off + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int kstep = kUmmaBlockK * p.ksub;                  // K elements per ring stage
+  const int kstep = TF32 ? kUmmaBlockK / 2 : kUmmaBlockK * p.ksub;   // K elements per ring stage (128-byte rows)
   const int kblocks = (p.K + kstep - 1) / kstep;
+  // 3xTF32: the tensor core truncates the fp32 accumulator once per instruction, a bias that grows
+  // with the number of instructions in a chain (about 7e-9 K relative).  So a tile's K range is cut
+  // into chunks of p.chunk_blocks k-blocks; each chunk is accumulated in tensor memory on its own and
+  // the epilogue warps add the chunks up in registers with ordinary rounded fp32 additions.
+  const int chunk_blocks = TF32 ? p.chunk_blocks : kblocks;
   const int rank = PAIR ? (int)cluster_ctarank() : 0;      // 0 = leader
   // work units are dealt round-robin to CTAs (PAIR: to clusters)
   const long long unit0 = PAIR ? (long long)(blockIdx.x >> 1) : (long long)blockIdx.x;
@@ -374,13 +434,13 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
           // The sub-blocks of a stage are adjacent in K: consecutive requests for the same matrix
           // rows ask the DRAM for neighbouring 128-byte lines (out-of-range sub-blocks read as zero).
           for (int j = 0; j < p.ksub; ++j) {
-            const int k0 = kb * kstep + j * kUmmaBlockK;
+            const int k0 = kb * kstep + j * (TF32 ? p.k_plane : kUmmaBlockK);
             const uint32_t dst = xs + (uint32_t)(j * L.sub_bytes) + L.x_bytes;
             if constexpr (PAIR) tma_load_3d_pair(dst, &tmap_w, k0, c.n0 + rank * w_rows, c.bt, full_bar(s));
             else tma_load_3d(dst, &tmap_w, k0, c.n0, c.bt, full_bar(s));
           }
           for (int j = 0; j < p.ksub; ++j) {
-            const int k0 = kb * kstep + j * kUmmaBlockK;
+            const int k0 = kb * kstep + j * (TF32 ? p.k_plane : kUmmaBlockK);
             const uint32_t dst = xs + (uint32_t)(j * L.sub_bytes);
             if constexpr (PAIR) tma_load_3d_pair(dst, &tmap_x, k0, c.m0, c.bt, full_bar(s));
             else tma_load_3d(dst, &tmap_x, k0, c.m0, c.bt, full_bar(s));
@@ -403,21 +463,37 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
   } else if (warp == 1) {
     // ================================================================ MMA issuer (the leader CTA of a pair)
     if (lane == 0 && rank == 0) {
-      const uint32_t idesc = make_idesc(PAIR ? 2 * kUmmaTileM : kUmmaTileM, p.tile_n);
-      uint32_t it = 0, tcount = 0;
+      const uint32_t idesc = make_idesc(PAIR ? 2 * kUmmaTileM : kUmmaTileM, p.tile_n, TF32);
+      uint32_t it = 0, tcount = 0;       // tcount counts accumulator hand-overs: tiles, or K chunks of tiles (3xTF32)
       bool ok = true;
-      for (long long t = unit0; t < p.num_tiles && ok; t += unit_step, ++tcount) {
+      for (long long t = unit0; t < p.num_tiles && ok; t += unit_step)
+       for (int kb0 = 0; kb0 < kblocks && ok; kb0 += chunk_blocks, ++tcount) {
         const uint32_t buf = tcount & 1u, aph = (tcount >> 1) & 1u;
         if (!(ok = mbar_wait(tmem_empty_bar(buf), aph ^ 1u, abort_flag, p.status))) break;
         tcgen05_fence_after();
         const uint32_t d = tmem_base + buf * 256u;
-        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+        const int kb1 = kb0 + chunk_blocks < kblocks ? kb0 + chunk_blocks : kblocks;
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % p.stages;
           const uint32_t ph = (it / p.stages) & 1u;
           if (!(ok = mbar_wait(full_bar(s), ph, abort_flag, p.status))) break;
           tcgen05_fence_after();
           const uint32_t xs = base + (uint32_t)(s * L.stage_bytes);
-          for (int j = 0; j < p.ksub; ++j) {
+          if constexpr (TF32) {
+            const uint64_t a_hi = make_smem_desc(xs), b_hi = make_smem_desc(xs + L.x_bytes);
+            const uint64_t a_lo = make_smem_desc(xs + (uint32_t)L.sub_bytes), b_lo = make_smem_desc(xs + (uint32_t)L.sub_bytes + L.x_bytes);
+#pragma unroll
+            for (int pr = 0; pr < 3; ++pr) {               // the two small products first, then hi * hi
+              const uint64_t a0 = pr == 0 ? a_lo : a_hi, b0 = pr == 1 ? b_lo : b_hi;
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {                // 8 tf32 = 32 bytes = 2 descriptor address units
+                const uint32_t acc = ((kb - kb0) | pr | k) != 0 ? 1u : 0u;
+                if constexpr (PAIR) tcgen05_mma_tf32_pair(d, a0 + 2u * k, b0 + 2u * k, idesc, acc);
+                else tcgen05_mma_tf32(d, a0 + 2u * k, b0 + 2u * k, idesc, acc);
+              }
+            }
+          }
+          for (int j = 0; !TF32 && j < p.ksub; ++j) {
             const uint64_t a0 = make_smem_desc(xs + (uint32_t)(j * L.sub_bytes));
             const uint64_t b0 = make_smem_desc(xs + (uint32_t)(j * L.sub_bytes) + L.x_bytes);
 #pragma unroll
@@ -447,7 +523,6 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
     bool ok = true;
     for (long long t = unit0; t < p.num_tiles && ok; t += unit_step, ++tcount) {
       const TileCoord c = tile_coord(t, p, rank);
-      const uint32_t buf = tcount & 1u, aph = (tcount >> 1) & 1u;
       // stage the bias and scale of this warp's columns in its own slice of shared memory
       for (int i = lane; i < c_end - c_begin; i += 32) {
         const int n = c.n0 + c_begin + i;
@@ -461,26 +536,89 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
         if constexpr (SC) scale_s[i] = V::kFoldLog2e ? s * kLog2e : s;
       }
       __syncwarp();
+      const int m = c.m0 + quad * 32 + lane;
+      const bool row_ok = m < p.M;
+      const int n_valid = p.N - c.n0;       // columns of this tile inside the matrix (may exceed tile_n)
+      const int c_lim = c_end < n_valid ? c_end : n_valid;   // a multiple of 8 (fp32: of 4)
+      uint32_t ra[kChunk], rb[kChunk];
+      float y[kChunk];
+      // 3xTF32: the sums of this thread's (at most 128) columns over the K chunks seen so far
+      float S[TF32 ? 8 * kChunk : 1];
+      if constexpr (TF32) {
+#pragma unroll
+        for (int i = 0; i < 8 * kChunk; ++i) S[i] = 0.0f;
+        // every chunk but the last: add the chunk's accumulator to S and hand the buffer back
+        for (int kb0 = 0; kb0 + chunk_blocks < kblocks; kb0 += chunk_blocks, ++tcount) {
+          const uint32_t cbuf = tcount & 1u;
+          ok = __all_sync(0xffffffffu, mbar_wait(tmem_full_bar(cbuf), (tcount >> 1) & 1u, abort_flag, p.status));
+          if (!ok) break;
+          tcgen05_fence_after();
+          const uint32_t ca = tmem_base + ((uint32_t)(quad * 32) << 16) + cbuf * 256u;
+#pragma unroll
+          for (int q = 0; q < 8; q += 2) {
+            const int cc = c_begin + kChunk * q;
+            if (cc < c_lim) {
+              const bool second = cc + kChunk < c_lim;
+              tcgen05_ld16_issue(ca + cc, ra);
+              if (second) tcgen05_ld16_issue(ca + cc + kChunk, rb);
+              tcgen05_wait_ld();
+#pragma unroll
+              for (int j = 0; j < kChunk; ++j) S[kChunk * q + j] += __uint_as_float(ra[j]);
+              if (second) {
+#pragma unroll
+                for (int j = 0; j < kChunk; ++j) S[kChunk * (q + 1) + j] += __uint_as_float(rb[j]);
+              }
+            }
+          }
+          tcgen05_fence_before();
+          __syncwarp();
+          if (lane == 0) {
+            if constexpr (PAIR) mbar_arrive_leader(tmem_empty_bar(cbuf)); else mbar_arrive(tmem_empty_bar(cbuf));
+          }
+        }
+        if (!ok) break;
+      }
+      const uint32_t buf = tcount & 1u, aph = (tcount >> 1) & 1u;
       ok = __all_sync(0xffffffffu, mbar_wait(tmem_full_bar(buf), aph, abort_flag, p.status));
       if (!ok) break;
       tcgen05_fence_after();
-
-      const int m = c.m0 + quad * 32 + lane;
-      const bool row_ok = m < p.M;
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * 256u;
-      __nv_bfloat16* yrow = static_cast<__nv_bfloat16*>(p.Y) + (long long)c.bt * p.bsy + (long long)m * p.ldy + c.n0;
-      const int n_valid = p.N - c.n0;       // columns of this tile inside the matrix (may exceed tile_n)
-      const int c_lim = c_end < n_valid ? c_end : n_valid;   // a multiple of 8
+      using OutT = typename std::conditional<TF32, float, __nv_bfloat16>::type;
+      OutT* yrow = static_cast<OutT*>(p.Y) + (long long)c.bt * p.bsy + (long long)m * p.ldy + c.n0;
+      // is column j of a 16-column chunk with nv real columns inside the matrix?  (bf16: N is a multiple
+      // of 8, so a ragged chunk has exactly 8; fp32: a multiple of 4)
+      auto real = [](int j, int nv) { return TF32 ? j < nv : (j < 8 || nv >= kChunk); };
+      auto store16 = [&](int cc, const float* yy, int nv) {
+        if constexpr (TF32) store_f32x16(yrow + cc, yy, nv);
+        else store_bf16x16(yrow + cc, yy, nv >= kChunk);
+      };
 
       float r0 = -CUDART_INF_F, r1 = 0.0f;  // (max, sum) or (max in log2 units, sum of 2^(t - max))
-      uint32_t ra[kChunk], rb[kChunk];
-      float y[kChunk];
 
       // Walks this warp's columns 32 at a time: both loads are issued before the single wait.
       // f(y, cc, nv): y = epilogue values of columns cc .. cc+15, nv = how many of them are real
       // (16 or more, or exactly 8 in the last chunk of a matrix whose N is not a multiple of 16).
+      bool folded = false;                  // 3xTF32: has the last chunk been added to S yet?
       auto sweep = [&](auto&& f) {
-        for (int cc = c_begin; cc < c_lim; cc += 2 * kChunk) {
+        if constexpr (TF32) {
+          // fixed trip count and static indices keep S in registers
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const int cc = c_begin + kChunk * q;
+            if (cc < c_lim) {
+              if (!folded) {
+                tcgen05_ld16_issue(taddr + cc, ra);
+                tcgen05_wait_ld();
+#pragma unroll
+                for (int j = 0; j < kChunk; ++j) S[kChunk * q + j] += __uint_as_float(ra[j]);
+              }
+              apply16f<ACT, SC>(S + kChunk * q, bias_s + kChunk * q, scale_s + kChunk * q, y);
+              f(y, cc, c_lim - cc);
+            }
+          }
+          folded = true;
+        }
+        for (int cc = c_begin; !TF32 && cc < c_lim; cc += 2 * kChunk) {
           const bool second = cc + kChunk < c_lim;
           tcgen05_ld16_issue(taddr + cc, ra);
           if (second) tcgen05_ld16_issue(taddr + cc + kChunk, rb);
@@ -498,22 +636,21 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
         // pass A: row maximum over this warp's columns (log2 units)
         sweep([&](float* yy, int, int nv) {
 #pragma unroll
-          for (int j = 0; j < kChunk; ++j) if (j < 8 || nv >= kChunk) r0 = fmaxf(r0, yy[j]);
+          for (int j = 0; j < kChunk; ++j) if (real(j, nv)) r0 = fmaxf(r0, yy[j]);
         });
         // pass B: exponentials relative to that maximum, their sum, and the bf16 store
         sweep([&](float* yy, int cc, int nv) {
 #pragma unroll
           for (int j = 0; j < kChunk; ++j) {
-            yy[j] = (j < 8 || nv >= kChunk) ? ex2(yy[j] - r0) : 0.0f;
+            yy[j] = real(j, nv) ? ex2(yy[j] - r0) : 0.0f;
             r1 += yy[j];
           }
-          if (row_ok) store_bf16x16(yrow + cc, yy, nv >= kChunk);
+          if (row_ok) store16(cc, yy, nv);
         });
       } else {
         sweep([&](float* yy, int cc, int nv) {
-          const bool full = nv >= kChunk;
           if constexpr (V::kStoreY) {
-            if (row_ok) store_bf16x16(yrow + cc, yy, full);
+            if (row_ok) store16(cc, yy, nv);
           }
           if constexpr (V::kExp) {
             if constexpr (V::kStoreY) {
@@ -522,16 +659,16 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
             }
             float cm = -CUDART_INF_F;
 #pragma unroll
-            for (int j = 0; j < kChunk; ++j) if (j < 8 || full) cm = fmaxf(cm, yy[j]);
+            for (int j = 0; j < kChunk; ++j) if (real(j, nv)) cm = fmaxf(cm, yy[j]);
             const float mn = fmaxf(r0, cm);
             float l = 0.0f;
 #pragma unroll
-            for (int j = 0; j < kChunk; ++j) if (j < 8 || full) l += ex2(yy[j] - mn);
+            for (int j = 0; j < kChunk; ++j) if (real(j, nv)) l += ex2(yy[j] - mn);
             r1 = fmaf(r1, ex2(r0 - mn), l);
             r0 = mn;
           } else {
 #pragma unroll
-            for (int j = 0; j < kChunk; ++j) if (j < 8 || full) { r0 = fmaxf(r0, yy[j]); r1 += yy[j]; }
+            for (int j = 0; j < kChunk; ++j) if (real(j, nv)) { r0 = fmaxf(r0, yy[j]); r1 += yy[j]; }
           }
         });
       }
@@ -578,18 +715,25 @@ cudaError_t launch_one(const Params& p, const CUtensorMap& tx, const CUtensorMap
   attr[1].val.clusterDim.y = 1;
   attr[1].val.clusterDim.z = 1;
   cfg.attrs = attr;
+  const bool tf32 = p.dtype == FGR_F32;
   if (p.cta_pair == 2) {
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, umma_kernel<ACT, SC, RED, WY, true>, tx, tw, p);
+    if (tf32) return cudaLaunchKernelEx(&cfg, umma_kernel<ACT, SC, RED, WY, true, true>, tx, tw, p);
+    return cudaLaunchKernelEx(&cfg, umma_kernel<ACT, SC, RED, WY, true, false>, tx, tw, p);
   }
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, umma_kernel<ACT, SC, RED, WY, false>, tx, tw, p);
+  if (tf32) return cudaLaunchKernelEx(&cfg, umma_kernel<ACT, SC, RED, WY, false, true>, tx, tw, p);
+  return cudaLaunchKernelEx(&cfg, umma_kernel<ACT, SC, RED, WY, false, false>, tx, tw, p);
 }
 template <int ACT, bool SC, int RED, bool WY>
 cudaError_t prepare_one() {
-  cudaError_t e = cudaFuncSetAttribute(umma_kernel<ACT, SC, RED, WY, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+  cudaError_t e = cudaFuncSetAttribute(umma_kernel<ACT, SC, RED, WY, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(umma_kernel<ACT, SC, RED, WY, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+    e = cudaFuncSetAttribute(umma_kernel<ACT, SC, RED, WY, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(umma_kernel<ACT, SC, RED, WY, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(umma_kernel<ACT, SC, RED, WY, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
   return e;
 }
 
