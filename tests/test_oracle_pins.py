@@ -390,3 +390,41 @@ def test_further_activations_in_the_chain(act, fn):
     y = fn(torch.from_numpy(X).double() @ torch.from_numpy(W).double().T + torch.from_numpy(b).double()) * -0.5
     np.testing.assert_allclose(Y, y.numpy(), rtol=1e-13, atol=1e-15)
     np.testing.assert_allclose(out[:, 0], torch.logsumexp(y, 1).numpy(), rtol=1e-13)
+
+
+# ---------------------------------------------------------------- 1-D convolution as window matrix
+def test_conv1d_windows_hand_example():
+    # x [L=4, C=2] = rows (1,2) (3,4) (5,6) (7,8); taps = 2 -> windows (1,2,3,4) (3,4,5,6) (5,6,7,8)
+    x = np.arange(1, 9, dtype=np.float32).reshape(1, 4, 2)
+    A = oracle.conv1d_windows(x, 2)
+    assert A.shape == (1, 3, 4)
+    np.testing.assert_array_equal(A[0], [[1, 2, 3, 4], [3, 4, 5, 6], [5, 6, 7, 8]])
+    # one filter w[r, c] = ((1, 0), (0, -1)): z[l] = x[l, 0] - x[l + 1, 1] = 1 - 4, 3 - 6, 5 - 8
+    w = np.array([[[1, 0], [0, -1]]], dtype=np.float32).reshape(1, 1, 4)
+    Y, out, _ = _run(A, w, None, None, reduce=oracle.RED_MAXSUM)
+    np.testing.assert_array_equal(Y.ravel(), [-3, -3, -3])
+    np.testing.assert_array_equal(oracle.conv1d_windows(x, 1), x)          # one tap: the plain linear layer
+    np.testing.assert_array_equal(oracle.conv1d_windows(x, 4)[0], x.reshape(1, 8))
+    with pytest.raises(ValueError):
+        oracle.conv1d_windows(x, 5)
+
+
+def test_conv1d_matches_library_fp64_and_shift_kernel():
+    B, L, C, N, R = 2, 19, 6, 5, 4
+    x = _rand((B, L, C), 51)
+    w = _rand((N, R, C), 52, tid=8)
+    b = gi.uniform(53, 3, N, -1, 1)
+    A = oracle.conv1d_windows(x, R)
+    Y, out, _ = oracle.run(A, np.broadcast_to(w.reshape(1, N, R * C), (B, N, R * C)).copy(), b, None, dtype=oracle.F32,
+                           act=oracle.ACT_RELU, scale_kind=oracle.SCALE_NONE, reduce=oracle.RED_LSE)
+    # library routine: torch's conv1d takes [B, C, L] and weights [N, C, R]
+    ref = torch.nn.functional.conv1d(torch.from_numpy(x).double().permute(0, 2, 1), torch.from_numpy(w).double().permute(0, 2, 1),
+                                     torch.from_numpy(b).double()).relu().permute(0, 2, 1).reshape(B * (L - R + 1), N)
+    np.testing.assert_allclose(Y, ref.numpy(), rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(out[:, 0], torch.logsumexp(ref, 1).numpy(), rtol=1e-13)
+    # a filter that is 1 at (tap r0, channel c0) and 0 elsewhere copies the shifted input: z[b, l] = x[b, l + r0, c0]
+    r0, c0 = 2, 3
+    d = np.zeros((1, 1, R * C), np.float32)
+    d[0, 0, r0 * C + c0] = 1.0
+    Yd, _, _ = oracle.run(A[:1], d, None, None, dtype=oracle.F32, act=oracle.ACT_NONE, scale_kind=oracle.SCALE_NONE, reduce=oracle.RED_MAXSUM)
+    np.testing.assert_array_equal(Yd.ravel(), x[0, r0:r0 + L - R + 1, c0].astype(np.float64))
