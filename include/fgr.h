@@ -97,6 +97,18 @@ typedef struct fgr_desc {
   int32_t force_cta_pair;  /* 0 = automatic; 1 = every CTA alone (128-row tiles); 2 = clusters of two CTAs
                               sharing 256-row tiles (tcgen05 cta_group::2; needs tile_n % 32 == 0) */
   int32_t force_ksub;      /* 0 = automatic; else 1, 2 or 4: 64-wide K sub-blocks per shared-memory ring stage */
+  int32_t conv_taps;       /* 0 or 1: plain GEMM.  R > 1: 1-D convolution as an implicit GEMM (the operator category
+                              "convolution", Section 1 and Section 4.1; 1-D is the paper's case study, Section 4.4).
+                              X is then the channels-last input [batch, L, C] with L = M + R - 1 and C = K / R,
+                              W the filters [batch, N, R * C] (tap-major, channel-minor), stride 1, no padding:
+                                z[b, l, n] = sum_r sum_c X[b, l + r, c] * W[n, r * C + c],   l = 0 .. M - 1.
+                              Output row l of the GEMM reads the K = R * C contiguous elements that start at
+                              X[b, l, 0], so the rows of the implicit matrix overlap: ldx is C (0 or C; channel
+                              padding is not supported) and bsx defaults to L * C; nothing is copied or unfolded.  K % R == 0 and C a multiple of 8 (bf16)
+                              / 4 (fp32).  fgr_run_static takes plain GEMMs only. */
+  int32_t w_shared;        /* 0: W is [batch, N, K] (one weight matrix per batch element).  1: W is one [N, K] matrix
+                              used by every batch element (bsw is ignored) - a filter bank shared by all signals of
+                              a convolution, or one linear layer applied to a batch of inputs */
 } fgr_desc;
 
 /* What fgr_plan / fgr_create decided; plain host data, for callers, tests and benchmarks. */

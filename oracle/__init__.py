@@ -81,7 +81,8 @@ def run(X, W, bias, scale_vec, *, dtype, act, scale_kind, reduce, scale=1.0, bia
         rows=None, want_y=True, nthreads=0):
     """Evaluates the operator's definition in fp64.
 
-    X [batch, M, K] and W [batch, N, K] (2-D arrays are taken as batch 1): fp32 values
+    X [batch, M, K] and W [batch, N, K] (2-D arrays are taken as batch 1; a W of batch 1 is used for
+    every batch element of X): fp32 values
     (``dtype == F32``) or uint16 bf16 bit patterns (``dtype == BF16``).  ``bias`` fp32 [N]
     (or [batch, N] with ``bias_per_batch``) or None; ``scale_vec`` fp32 [N] or None.
     ``rows``: global row indices (bt * M + m) to evaluate; None = all rows.
@@ -99,6 +100,8 @@ def run(X, W, bias, scale_vec, *, dtype, act, scale_kind, reduce, scale=1.0, bia
     if W.ndim == 2:
         W = W[None]
     batch, M, K = X.shape
+    if W.shape[0] == 1 and batch > 1:          # one weight matrix shared by every batch element
+        W = np.ascontiguousarray(np.broadcast_to(W, (batch,) + W.shape[1:]))
     if W.shape[0] != batch or W.shape[2] != K:
         raise ValueError("shape mismatch between X %s and W %s" % (X.shape, W.shape))
     N = W.shape[1]

@@ -56,11 +56,12 @@ struct Resolved { long long ldx, ldw, ldy, bsx, bsw, bsy; };
 
 Resolved resolve_strides(const fgr_desc& d) {
   Resolved r;
-  r.ldx = d.ldx ? d.ldx : d.K;
+  const int taps = d.conv_taps > 1 ? d.conv_taps : 1;   // 1-D convolution: rows of the implicit matrix overlap
+  r.ldx = d.ldx ? d.ldx : d.K / taps;
   r.ldw = d.ldw ? d.ldw : d.K;
   r.ldy = d.ldy ? d.ldy : d.N;
-  r.bsx = d.bsx ? d.bsx : (long long)d.M * r.ldx;
-  r.bsw = d.bsw ? d.bsw : (long long)d.N * r.ldw;
+  r.bsx = d.bsx ? d.bsx : (long long)(d.M + taps - 1) * r.ldx;
+  r.bsw = d.w_shared ? 0 : (d.bsw ? d.bsw : (long long)d.N * r.ldw);   // shared W: every batch reads the same matrix
   r.bsy = d.bsy ? d.bsy : (long long)d.M * r.ldy;
   return r;
 }
@@ -81,10 +82,15 @@ int validate(const fgr_desc* d) {
   if (d->ldx < 0 || d->ldw < 0 || d->ldy < 0 || d->bsx < 0 || d->bsw < 0 || d->bsy < 0) return FGR_ERR_INVALID_ARG;
   const int g = 16 / elem_bytes(d->dtype);   // elements per 16 bytes
   if (d->K % g || d->N % g) return FGR_ERR_UNSUPPORTED;
+  if (d->conv_taps < 0 || (d->w_shared != 0 && d->w_shared != 1)) return FGR_ERR_INVALID_ARG;
+  const int taps = d->conv_taps > 1 ? d->conv_taps : 1;
+  if (d->K % taps) return FGR_ERR_INVALID_ARG;
+  if ((d->K / taps) % g) return FGR_ERR_UNSUPPORTED;
   const Resolved r = resolve_strides(*d);
-  if (r.ldx < d->K || r.ldw < d->K || r.ldy < d->N) return FGR_ERR_INVALID_ARG;
+  if (r.ldx < d->K / taps || r.ldw < d->K || r.ldy < d->N) return FGR_ERR_INVALID_ARG;
+  if (taps > 1 && r.ldx != d->K / taps) return FGR_ERR_UNSUPPORTED;   // a window must be K contiguous elements
   if (r.ldx % g || r.ldw % g || r.ldy % g || r.bsx % g || r.bsw % g || r.bsy % g) return FGR_ERR_UNSUPPORTED;
-  if (d->batch > 1 && (r.bsx < (long long)(d->M - 1) * r.ldx + d->K || r.bsw < (long long)(d->N - 1) * r.ldw + d->K ||
+  if (d->batch > 1 && (r.bsx < (long long)(d->M - 1) * r.ldx + d->K || (!d->w_shared && r.bsw < (long long)(d->N - 1) * r.ldw + d->K) ||
                        r.bsy < (long long)(d->M - 1) * r.ldy + d->N))
     return FGR_ERR_INVALID_ARG;
   if ((long long)d->batch * d->M > (1LL << 31) - 1) return FGR_ERR_UNSUPPORTED;
@@ -96,7 +102,8 @@ int validate(const fgr_desc* d) {
 
 double min_bytes(const fgr_desc& d) {
   const double e = elem_bytes(d.dtype);
-  double b = (double)d.batch * ((double)d.M * d.K + (double)d.N * d.K) * e;
+  const int taps = d.conv_taps > 1 ? d.conv_taps : 1;   // a convolution's input is read once, not once per tap
+  double b = ((double)d.batch * (d.M + taps - 1) * (d.K / taps) + (double)(d.w_shared ? 1 : d.batch) * d.N * d.K) * e;
   b += 4.0 * d.N * (d.bias_per_batch ? d.batch : 1);   // bias (counted whether or not one is passed)
   if (d.scale_kind == FGR_SCALE_PER_COLUMN) b += 4.0 * d.N;
   if (d.write_y || d.reduce == FGR_RED_SOFTMAX) b += (double)d.batch * d.M * d.N * e;
@@ -147,6 +154,7 @@ int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
   p.batch = d.batch; p.M = d.M; p.N = d.N; p.K = d.K;
   p.dtype = d.dtype; p.act = d.act; p.scale_kind = d.scale_kind; p.reduce = d.reduce;
   p.write_y = d.write_y; p.bias_per_batch = d.bias_per_batch; p.scale = d.scale;
+  p.w_shared = d.w_shared;
   p.ldx = r.ldx; p.ldw = r.ldw; p.ldy = r.ldy; p.bsx = r.bsx; p.bsw = r.bsw; p.bsy = r.bsy;
 
   if (path == FGR_PATH_SIMT_GEMV) {
@@ -234,7 +242,7 @@ int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
   pi.workspace_bytes = (uint64_t)kStatusBytes + (uint64_t)d.batch * d.M * p.parts_per_row * 8ull;
   if (tf32)   // the hi / lo planes of X and W follow the partial pairs, each on a 256-byte boundary
     pi.workspace_bytes = align256(align256((size_t)pi.workspace_bytes) + (size_t)d.batch * d.M * 2 * p.k_plane * 4) +
-                         (uint64_t)d.batch * d.N * 2 * p.k_plane * 4;
+                         (uint64_t)(d.w_shared ? 1 : d.batch) * d.N * 2 * p.k_plane * 4;
   *info = pi;
   if (pp) *pp = p;
   return FGR_OK;
@@ -380,7 +388,7 @@ int fgr_run(fgr_handle* h, const void* X, const void* W, const float* bias, cons
     xp = reinterpret_cast<float*>(wsb + x_off);
     wp = reinterpret_cast<float*>(wsb + w_off);
     e = launch_split_tf32(static_cast<const float*>(X), xp, d.batch, d.M, d.K, p.ldx, p.bsx, p.k_plane, stream);
-    if (e == cudaSuccess) e = launch_split_tf32(static_cast<const float*>(W), wp, d.batch, d.N, d.K, p.ldw, p.bsw, p.k_plane, stream);
+    if (e == cudaSuccess) e = launch_split_tf32(static_cast<const float*>(W), wp, d.w_shared ? 1 : d.batch, d.N, d.K, p.ldw, p.bsw, p.k_plane, stream);
   }
   if (e == cudaSuccess && ev0) e = cudaEventRecord(ev0, stream);
   if (e == cudaSuccess) {
@@ -393,7 +401,7 @@ int fgr_run(fgr_handle* h, const void* X, const void* W, const float* bias, cons
       if (workspace != h->cached_x) {   // the tensor maps describe the planes, which live in the workspace
         const long long ldp = 2LL * p.k_plane;
         rc = encode_operand(&h->tmap_x, xp, (int)ldp, d.M, d.batch, ldp, (long long)d.M * ldp, kUmmaTileM, true);
-        if (rc == FGR_OK) rc = encode_operand(&h->tmap_w, wp, (int)ldp, d.N, d.batch, ldp, (long long)d.N * ldp, p.tile_n / p.cta_pair, true);
+        if (rc == FGR_OK) rc = encode_operand(&h->tmap_w, wp, (int)ldp, d.N, d.w_shared ? 1 : d.batch, ldp, (long long)d.N * ldp, p.tile_n / p.cta_pair, true);
         h->cached_x = rc == FGR_OK ? workspace : nullptr;
       }
       if (rc == FGR_OK && e == cudaSuccess) e = launch_umma(p, &h->tmap_x, &h->tmap_w, h->plan.grid, h->plan.smem_bytes, stream);
@@ -403,7 +411,7 @@ int fgr_run(fgr_handle* h, const void* X, const void* W, const float* bias, cons
         h->cached_x = rc == FGR_OK ? X : nullptr;
       }
       if (rc == FGR_OK && W != h->cached_w) {
-        rc = encode_operand(&h->tmap_w, W, d.K, d.N, d.batch, p.ldw, p.bsw, p.tile_n / p.cta_pair);
+        rc = encode_operand(&h->tmap_w, W, d.K, d.N, d.w_shared ? 1 : d.batch, p.ldw, p.bsw, p.tile_n / p.cta_pair);
         h->cached_w = rc == FGR_OK ? W : nullptr;
       }
       if (rc == FGR_OK) e = launch_umma(p, &h->tmap_x, &h->tmap_w, h->plan.grid, h->plan.smem_bytes, stream);

@@ -40,6 +40,7 @@ struct Params {
   int ksub;            // tcgen05 paths: 64-wide K sub-blocks per ring stage (1, 2 or 4)
   int cta_pair;        // tcgen05 paths: 1 = each CTA works alone, 2 = clusters of two CTAs share 256-row tiles
   int k_plane;         // 3xTF32 path: K rounded up to 32 = width of the hi plane (the lo plane follows it)
+  int w_shared;        // 1: W is one [N, K] matrix used by every batch element (bsw = 0)
   int chunk_blocks;    // 3xTF32 path: 32-wide k-blocks accumulated in tensor memory before the epilogue adds them up
 };
 

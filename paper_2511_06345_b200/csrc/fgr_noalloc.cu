@@ -42,6 +42,7 @@ int fgr_run_static(const fgr_desc* desc, const void* X, const void* W, const flo
   fgr_plan_info plan;
   int rc = fgr_plan(&d, 0, &plan);
   if (rc != FGR_OK) return rc;
+  if (d.conv_taps > 1) return FGR_ERR_UNSUPPORTED;   // plain GEMMs only
   const unsigned long long need = (unsigned long long)d.batch * d.M * plan.parts_per_row * 8ull;
   if (need > kScratchBytes) return FGR_ERR_WORKSPACE;   // the fixed scratch cannot hold this problem's partial pairs
 
@@ -76,7 +77,8 @@ int fgr_run_static(const fgr_desc* desc, const void* X, const void* W, const flo
     p.ldw = d.ldw ? d.ldw : d.K;
     p.ldy = d.ldy ? d.ldy : d.N;
     p.bsx = d.bsx ? d.bsx : (long long)d.M * p.ldx;
-    p.bsw = d.bsw ? d.bsw : (long long)d.N * p.ldw;
+    p.bsw = d.w_shared ? 0 : (d.bsw ? d.bsw : (long long)d.N * p.ldw);
+    p.w_shared = d.w_shared;
     p.bsy = d.bsy ? d.bsy : (long long)d.M * p.ldy;
     p.X = X; p.W = W; p.bias = bias; p.scale_vec = scale_vec; p.Y = Y; p.out = out;
     p.parts = g_scratch_addr[d.device];   // every pair the second kernel reads is written by the first

@@ -436,8 +436,8 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
           for (int j = 0; j < p.ksub; ++j) {
             const int k0 = kb * kstep + j * (TF32 ? p.k_plane : kUmmaBlockK);
             const uint32_t dst = xs + (uint32_t)(j * L.sub_bytes) + L.x_bytes;
-            if constexpr (PAIR) tma_load_3d_pair(dst, &tmap_w, k0, c.n0 + rank * w_rows, c.bt, full_bar(s));
-            else tma_load_3d(dst, &tmap_w, k0, c.n0, c.bt, full_bar(s));
+            if constexpr (PAIR) tma_load_3d_pair(dst, &tmap_w, k0, c.n0 + rank * w_rows, p.w_shared ? 0 : c.bt, full_bar(s));
+            else tma_load_3d(dst, &tmap_w, k0, c.n0, p.w_shared ? 0 : c.bt, full_bar(s));
           }
           for (int j = 0; j < p.ksub; ++j) {
             const int k0 = kb * kstep + j * (TF32 ? p.k_plane : kUmmaBlockK);

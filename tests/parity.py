@@ -43,7 +43,8 @@ def run_gpu(p: gi.Problem, force_path=0, force_tile_n=0, device=0, tensors=None,
     out float64 [rows, w] or None, plan dict)."""
     op = fgr.FusedGemmReduce(p.batch, p.M, p.N, p.K, p.dtype, p.act, p.scale_kind, p.reduce, scale=p.scale,
                              write_y=p.write_y, bias_per_batch=p.bias_per_batch, device=device,
-                             force_path=force_path, force_tile_n=force_tile_n, force_cta_pair=force_cta_pair, force_ksub=force_ksub)
+                             force_path=force_path, force_tile_n=force_tile_n, force_cta_pair=force_cta_pair, force_ksub=force_ksub,
+                             conv_taps=p.conv_taps, w_shared=p.w_shared)
     X, W, b, s = tensors if tensors is not None else to_device(p, "cuda:%d" % device)
     for _ in range(repeat):
         Y, out = op(X, W, b, s)

@@ -261,3 +261,19 @@ def test_identity_weights(cuda_device):
     got = torch.from_numpy(ref).to(torch.bfloat16).float().numpy()
     np.testing.assert_array_equal(Y.astype(np.float32), got)
     compare(p, Y, out)
+
+
+def test_shared_weights_plain_gemm(cuda_device):
+    """w_shared = 1 without a convolution: one [N, K] weight matrix for a batch of inputs, on every path."""
+    for dtype, path in [(gi.DTYPE_BF16, fgr.FGR_PATH_UMMA_TILED), (gi.DTYPE_BF16, fgr.FGR_PATH_UMMA_STREAM_W),
+                        (gi.DTYPE_BF16, fgr.FGR_PATH_SIMT), (gi.DTYPE_F32, fgr.FGR_PATH_SIMT), (gi.DTYPE_F32, fgr.FGR_PATH_UMMA_TF32X3)]:
+        p = gi.make_problem("t", 3, 130, 264, 72, dtype, gi.ACT_RELU, gi.SCALE_NONE, gi.RED_MAX_SUMEXP, write_y=1, x_std=1.0,
+                            w_std=0.2, seed=31, w_shared=1)
+        assert p.W.shape == (1, 264, 72)
+        Y, out, plan = run_gpu(p, force_path=path)
+        assert plan["path"] == path
+        compare(p, Y, out, tcgen05=dtype == gi.DTYPE_BF16 and path != fgr.FGR_PATH_SIMT)
+    p = gi.make_problem("t", 3, 4, 264, 72, gi.DTYPE_BF16, gi.ACT_RELU, gi.SCALE_NONE, gi.RED_LSE, write_y=1, w_std=0.2, seed=32, w_shared=1)
+    Y, out, plan = run_gpu(p)
+    assert plan["path"] == fgr.FGR_PATH_SIMT_GEMV
+    compare(p, Y, out)
