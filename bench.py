@@ -31,7 +31,9 @@ METRIC = "fused GEMM+epilogue+rowreduce TFLOP/s (or GB/s) and % of roofline, 1 B
 HBM_BOUND = {"c4", "g2"}
 # extra workloads of the fused operator beside the five named ones: the skinny CUDA-core GEMV path
 EXTRA_CONFIGS = {"g2": ("c4", dict(M=2)),     # c4's shapes and epilogue with M = 2
-                 "f2": ("c2", dict(dtype=0))}  # c2's shapes and epilogue with fp32 inputs and outputs: the 3xTF32 path
+                 "f2": ("c2", dict(dtype=0)),  # c2's shapes and epilogue with fp32 inputs and outputs: the 3xTF32 path
+                 # 1-D convolution with c2's epilogue: 8 signals of 2051 x 512 channels, 4096 filters of 4 taps (shared)
+                 "v2": ("c2", dict(batch=8, M=2048, N=4096, K=2048, conv_taps=4, w_shared=1))}
 
 
 def make_cfg(name, **kw):
@@ -242,7 +244,8 @@ def run_ours(args):
         s["out"] = torch.empty((rows, p.out_width), dtype=torch.float32, device=dev) if p.out_width else None
 
     desc = fgr.make_desc(p.batch, p.M, p.N, p.K, p.dtype, p.act, p.scale_kind, p.reduce, scale=p.scale,
-                         write_y=p.write_y, bias_per_batch=p.bias_per_batch, device=local_rank)
+                         write_y=p.write_y, bias_per_batch=p.bias_per_batch, device=local_rank,
+                         conv_taps=p.conv_taps, w_shared=p.w_shared)
     h = fgr.fgr_create(desc)
     plan = fgr.fgr_get_plan(h)
     ws_bytes = fgr.fgr_workspace_bytes(h)
@@ -352,6 +355,7 @@ def run_ours(args):
             "config": {"workload": cfg, "batch": p.batch, "M": p.M, "N": p.N, "K": p.K,
                        "act": ["none", "relu", "gelu_tanh"][p.act], "scale": ["none", "scalar", "per_column"][p.scale_kind],
                        "reduce": ["lse", "softmax", "maxsum", "max_sumexp"][p.reduce], "write_y": int(need_y),
+                       "conv_taps": p.conv_taps, "w_shared": p.w_shared,
                        "path": fgr.fgr_path_name(plan.path), "tile": [plan.tile_m, plan.tile_n], "stages": plan.stages,
                        "grid": plan.grid, "l2": "rotating %d distinct input/output sets (%.0f MB > 126 MB L2)" % (rot, rot * set_bytes / 1e6),
                        "parallelism": "independent problems per GPU, no collective" if world > 1 else "1 GPU"},
