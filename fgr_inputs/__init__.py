@@ -39,6 +39,7 @@ DTYPE_F32, DTYPE_BF16 = 0, 1
 ACT_NONE, ACT_RELU, ACT_GELU_TANH, ACT_SIGMOID, ACT_TANH, ACT_SILU = 0, 1, 2, 3, 4, 5
 SCALE_NONE, SCALE_SCALAR, SCALE_PER_COLUMN = 0, 1, 2
 RED_LSE, RED_SOFTMAX, RED_MAXSUM, RED_MAX_SUMEXP = 0, 1, 2, 3
+RED_MEANVAR = 6
 
 
 def _mix64(z: np.ndarray) -> np.ndarray:
@@ -143,7 +144,7 @@ class Problem:
 
     @property
     def out_width(self) -> int:
-        return {RED_LSE: 1, RED_SOFTMAX: 0, RED_MAXSUM: 2, RED_MAX_SUMEXP: 2}[self.reduce]
+        return {RED_LSE: 1, RED_SOFTMAX: 0, RED_MAXSUM: 2, RED_MAX_SUMEXP: 2, RED_MEANVAR: 2}[self.reduce]
 
     @property
     def elem_bytes(self) -> int:

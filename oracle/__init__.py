@@ -22,6 +22,7 @@ ACT_NONE, ACT_RELU, ACT_GELU_TANH, ACT_SIGMOID, ACT_TANH, ACT_SILU = 0, 1, 2, 3,
 SCALE_NONE, SCALE_SCALAR, SCALE_PER_COLUMN = 0, 1, 2
 RED_LSE, RED_SOFTMAX, RED_MAXSUM, RED_MAX_SUMEXP = 0, 1, 2, 3
 RED_MAX, RED_SUM = 4, 5          # stand-alone reduction only
+RED_MEANVAR = 6                  # (mean, population variance) of y over N
 
 
 class _Problem(ctypes.Structure):
@@ -70,7 +71,7 @@ def act(kind: int, u: float) -> float:
 
 
 def out_width(reduce: int) -> int:
-    return {RED_LSE: 1, RED_SOFTMAX: 0, RED_MAXSUM: 2, RED_MAX_SUMEXP: 2}[reduce]
+    return {RED_LSE: 1, RED_SOFTMAX: 0, RED_MAXSUM: 2, RED_MAX_SUMEXP: 2, RED_MEANVAR: 2}[reduce]
 
 
 def _ptr(a):
@@ -180,7 +181,7 @@ def reduce_rows(A, *, dtype, kind):
         raise TypeError("A must be a 2-D %s array with contiguous rows" % want.__name__)
     M, N = A.shape
     lda = A.strides[0] // A.itemsize
-    w = {RED_LSE: 1, RED_SOFTMAX: 0, RED_MAXSUM: 2, RED_MAX_SUMEXP: 2, RED_MAX: 1, RED_SUM: 1}[kind]
+    w = {RED_LSE: 1, RED_SOFTMAX: 0, RED_MAXSUM: 2, RED_MAX_SUMEXP: 2, RED_MAX: 1, RED_SUM: 1, RED_MEANVAR: 2}[kind]
     P = np.empty((M, N), np.float64) if kind == RED_SOFTMAX else None
     out = np.empty((M, w) if w == 2 else (M,), np.float64) if w else None
     rc = lib().fgr_oracle_reduce_rows(M, N, dtype, kind, A.ctypes.data_as(ctypes.c_void_p), lda, _ptr(P), _ptr(out))

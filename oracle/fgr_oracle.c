@@ -22,6 +22,8 @@
  *   SOFTMAX    : P[m,n]   = exp(y - mx) / sum_n exp(y - mx)
  *   MAXSUM     : out[m,:] = ( mx , sum_n y )
  *   MAX_SUMEXP : out[m,:] = ( mx , sum_n exp(y - mx) )
+ *   MEANVAR    : out[m,:] = ( mu , (1/N) sum_n (y - mu)^2 ),  mu = (1/N) sum_n y
+ *                (the row statistics of a normalisation layer: population variance, two passes)
  *
  *   act: NONE a = u;  RELU a = max(u, 0);
  *        GELU_TANH a = 0.5 u (1 + tanh( sqrt(2/pi) (u + 0.044715 u^3) ))
@@ -49,7 +51,7 @@
 enum { ORC_F32 = 0, ORC_BF16 = 1 };
 enum { ORC_ACT_NONE = 0, ORC_ACT_RELU = 1, ORC_ACT_GELU_TANH = 2, ORC_ACT_SIGMOID = 3, ORC_ACT_TANH = 4, ORC_ACT_SILU = 5 };
 enum { ORC_SCALE_NONE = 0, ORC_SCALE_SCALAR = 1, ORC_SCALE_PER_COLUMN = 2 };
-enum { ORC_RED_LSE = 0, ORC_RED_SOFTMAX = 1, ORC_RED_MAXSUM = 2, ORC_RED_MAX_SUMEXP = 3 };
+enum { ORC_RED_LSE = 0, ORC_RED_SOFTMAX = 1, ORC_RED_MAXSUM = 2, ORC_RED_MAX_SUMEXP = 3, ORC_RED_MEANVAR = 6 };
 
 typedef struct {
   int32_t batch, M, N, K;
@@ -106,6 +108,14 @@ static void oracle_row(const fgr_oracle_problem* p, const void* X, const void* W
     else if (p->scale_kind == ORC_SCALE_PER_COLUMN) s = (double)scale_vec[n];
     y[n] = a * s;
   }
+  if (p->reduce == ORC_RED_MEANVAR) {
+    double sum = 0.0, dev = 0.0;
+    for (int64_t n = 0; n < N; ++n) sum += y[n];
+    const double mu = sum / (double)N;
+    for (int64_t n = 0; n < N; ++n) dev += (y[n] - mu) * (y[n] - mu);
+    if (red) { red[0] = mu; red[1] = dev / (double)N; }
+    return;
+  }
   double mx = y[0];
   for (int64_t n = 1; n < N; ++n) if (y[n] > mx) mx = y[n];
   if (p->reduce == ORC_RED_MAXSUM) {
@@ -122,7 +132,7 @@ static void oracle_row(const fgr_oracle_problem* p, const void* X, const void* W
 }
 
 static int out_width(int reduce) {
-  return reduce == ORC_RED_LSE ? 1 : reduce == ORC_RED_SOFTMAX ? 0 : 2;
+  return reduce == ORC_RED_LSE ? 1 : reduce == ORC_RED_SOFTMAX ? 0 : 2;   /* MAXSUM, MAX_SUMEXP, MEANVAR */
 }
 
 /*
@@ -139,7 +149,7 @@ int fgr_oracle_rows(const fgr_oracle_problem* p, const void* X, const void* W, c
   if (!p || !X || !W || nrows < 0) return -1;
   if (p->batch < 1 || p->M < 1 || p->N < 1 || p->K < 1) return -2;
   if (p->dtype != ORC_F32 && p->dtype != ORC_BF16) return -3;
-  if (p->act < 0 || p->act > 5 || p->scale_kind < 0 || p->scale_kind > 2 || p->reduce < 0 || p->reduce > 3) return -4;
+  if (p->act < 0 || p->act > 5 || p->scale_kind < 0 || p->scale_kind > 2 || p->reduce < 0 || (p->reduce > 3 && p->reduce != ORC_RED_MEANVAR)) return -4;
   if (p->scale_kind == ORC_SCALE_PER_COLUMN && !scale_vec) return -5;
   const int64_t total = (int64_t)p->batch * p->M;
   for (int64_t i = 0; i < nrows; ++i) {
@@ -178,6 +188,7 @@ int fgr_oracle_out_width(int reduce) { return out_width(reduce); }
  * "reduction" of Section 4.1, Datasets; the paper's GPU case study is a max reduction over a
  * dimension, Section 4.4.1).  Same four kinds as above, applied to y = A directly, plus
  *   kind 4 (MAX): out[m] = max_n A[m, n]          kind 5 (SUM): out[m] = sum_n A[m, n]
+ *   kind 6 (MEANVAR): out[m, :] = (mean, population variance) of row m, as above
  * P (SOFTMAX) and out are fp64; A is fp32 or bf16 bit patterns, row stride lda elements.
  * Returns 0, or a negative value on a bad argument.
  */
@@ -185,8 +196,16 @@ int fgr_oracle_reduce_rows(int32_t M, int32_t N, int32_t dtype, int32_t kind, co
                            double* P, double* out) {
   if (M < 1 || N < 1 || !A || lda < N) return -1;
   if (dtype != ORC_F32 && dtype != ORC_BF16) return -3;
-  if (kind < 0 || kind > 5) return -4;
+  if (kind < 0 || kind > 6) return -4;
   for (int64_t m = 0; m < M; ++m) {
+    if (kind == ORC_RED_MEANVAR) {
+      double s = 0.0, dev = 0.0;
+      for (int64_t n = 0; n < N; ++n) s += load_elem(A, dtype, m * lda + n);
+      const double mu = s / (double)N;
+      for (int64_t n = 0; n < N; ++n) { double v = load_elem(A, dtype, m * lda + n) - mu; dev += v * v; }
+      out[2 * m] = mu; out[2 * m + 1] = dev / (double)N;
+      continue;
+    }
     double mx = load_elem(A, dtype, m * lda);
     for (int64_t n = 1; n < N; ++n) { double v = load_elem(A, dtype, m * lda + n); if (v > mx) mx = v; }
     double sum = 0.0, l = 0.0;

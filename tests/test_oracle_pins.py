@@ -428,3 +428,62 @@ def test_conv1d_matches_library_fp64_and_shift_kernel():
     d[0, 0, r0 * C + c0] = 1.0
     Yd, _, _ = oracle.run(A[:1], d, None, None, dtype=oracle.F32, act=oracle.ACT_NONE, scale_kind=oracle.SCALE_NONE, reduce=oracle.RED_MAXSUM)
     np.testing.assert_array_equal(Yd.ravel(), x[0, r0:r0 + L - R + 1, c0].astype(np.float64))
+
+
+# ---------------------------------------------------------------- mean / variance over N
+def test_meanvar_closed_forms():
+    N = 12
+    # W = I, b = 0: y = X.  Row 0 constant (variance 0), row 1 the sequence 0 .. N-1: mean (N-1)/2, variance (N^2-1)/12
+    X = np.stack([np.full(N, 3.25, np.float32), np.arange(N, dtype=np.float32)])
+    _, out, _ = _run(X, np.eye(N, dtype=np.float32), None, None, reduce=oracle.RED_MEANVAR)
+    np.testing.assert_allclose(out, [[3.25, 0.0], [(N - 1) / 2, (N * N - 1) / 12]], rtol=0, atol=1e-15)
+    out2 = oracle.reduce_rows(X, dtype=oracle.F32, kind=oracle.RED_MEANVAR)[1]
+    np.testing.assert_array_equal(out2, out)
+    # two values a, b: mean (a+b)/2, variance ((a-b)/2)^2 -- a large common offset must not spoil it
+    A = np.array([[1.0e6 + 1.0, 1.0e6 + 3.0]], np.float32)
+    np.testing.assert_allclose(oracle.reduce_rows(A, dtype=oracle.F32, kind=oracle.RED_MEANVAR)[1], [[1.0e6 + 2.0, 1.0]], rtol=0, atol=0)
+
+
+def test_meanvar_matches_library_and_invariants():
+    X, W, b = _rand((7, 20), 61, std=2.0), _rand((33, 20), 61, tid=8), gi.uniform(61, 3, 33, -1, 1)
+    Y, out, _ = _run(X, W, b, None, act=oracle.ACT_GELU_TANH, reduce=oracle.RED_MEANVAR)
+    y = torch.nn.functional.gelu(torch.from_numpy(X).double() @ torch.from_numpy(W).double().T + torch.from_numpy(b).double(),
+                                 approximate="tanh")
+    np.testing.assert_allclose(Y, y.numpy(), rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(out[:, 0], y.mean(1).numpy(), rtol=1e-13)
+    np.testing.assert_allclose(out[:, 1], y.var(1, unbiased=False).numpy(), rtol=1e-12)
+    # tie to the (max, sum) kind: mean = sum / N
+    _, ms, _ = _run(X, W, b, None, act=oracle.ACT_GELU_TANH, reduce=oracle.RED_MAXSUM)
+    np.testing.assert_allclose(out[:, 0], ms[:, 1] / 33, rtol=1e-14)
+    # no activation: shifting every bias by c shifts the mean by c and leaves the variance; scaling by a scales it by a^2
+    _, o0, _ = _run(X, W, b, None, reduce=oracle.RED_MEANVAR)
+    _, o1, _ = _run(X, W, (b + 2.5).astype(np.float32), None, reduce=oracle.RED_MEANVAR)
+    np.testing.assert_allclose(o1[:, 0] - o0[:, 0], 2.5, atol=1e-6)
+    np.testing.assert_allclose(o1[:, 1], o0[:, 1], rtol=1e-6)
+    _, o2, _ = _run(X, W, b, None, scale_kind=oracle.SCALE_SCALAR, scale=-3.0, reduce=oracle.RED_MEANVAR)
+    np.testing.assert_allclose(o2[:, 0], -3.0 * o0[:, 0], rtol=1e-13)
+    np.testing.assert_allclose(o2[:, 1], 9.0 * o0[:, 1], rtol=1e-13)
+    assert (out[:, 1] >= 0).all()
+
+
+def test_meanvar_merge_of_slices_is_exact_identity():
+    """The pairwise update used to merge per-tile (mean, M2) pairs:  delta = mean_b - mean_a,
+    mean = mean_a + delta n_b / n,  M2 = M2_a + M2_b + delta^2 n_a n_b / n  reproduces the whole-row
+    statistics from any split of the row (checked in fp64 on the oracle's own output)."""
+    A = _rand((5, 200), 62, std=3.0) + 7.0
+    whole = oracle.reduce_rows(A.astype(np.float32), dtype=oracle.F32, kind=oracle.RED_MEANVAR)[1]
+    for cuts in ([64, 128, 192], [8], [100], [16, 24, 184]):
+        edges = [0] + cuts + [200]
+        n = 0.0
+        mean = np.zeros(5)
+        M2 = np.zeros(5)
+        for a, b in zip(edges, edges[1:]):
+            part = oracle.reduce_rows(np.ascontiguousarray(A[:, a:b].astype(np.float32)), dtype=oracle.F32, kind=oracle.RED_MEANVAR)[1]
+            nb = float(b - a)
+            delta = part[:, 0] - mean
+            tot = n + nb
+            mean = mean + delta * nb / tot
+            M2 = M2 + part[:, 1] * nb + delta * delta * n * nb / tot
+            n = tot
+        np.testing.assert_allclose(mean, whole[:, 0], rtol=1e-13)
+        np.testing.assert_allclose(M2 / n, whole[:, 1], rtol=1e-12)
