@@ -354,7 +354,7 @@ def run_ours(args):
             "dtype": "bf16" if b16 else ("tf32x3" if plan.path == fgr.FGR_PATH_UMMA_TF32X3 else "f32"), "data": "synthetic",
             "config": {"workload": cfg, "batch": p.batch, "M": p.M, "N": p.N, "K": p.K,
                        "act": ["none", "relu", "gelu_tanh"][p.act], "scale": ["none", "scalar", "per_column"][p.scale_kind],
-                       "reduce": ["lse", "softmax", "maxsum", "max_sumexp"][p.reduce], "write_y": int(need_y),
+                       "reduce": {0: "lse", 1: "softmax", 2: "maxsum", 3: "max_sumexp", 6: "meanvar"}[p.reduce], "write_y": int(need_y),
                        "conv_taps": p.conv_taps, "w_shared": p.w_shared,
                        "path": fgr.fgr_path_name(plan.path), "tile": [plan.tile_m, plan.tile_n], "stages": plan.stages,
                        "grid": plan.grid, "l2": "rotating %d distinct input/output sets (%.0f MB > 126 MB L2)" % (rot, rot * set_bytes / 1e6),
@@ -375,6 +375,7 @@ REDUCE_CONFIGS = {   # stand-alone row reduction of a bf16 matrix, the paper's G
     "r_max": dict(M=8192, N=8192, kind=4, name="max"),
     "r_lse": dict(M=8192, N=8192, kind=0, name="lse"),
     "r_softmax": dict(M=8192, N=8192, kind=1, name="softmax"),
+    "r_meanvar": dict(M=8192, N=8192, kind=6, name="meanvar"),
 }
 
 

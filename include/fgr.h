@@ -64,7 +64,11 @@ typedef enum { FGR_F32 = 0, FGR_BF16 = 1 } fgr_dtype;
 typedef enum { FGR_ACT_NONE = 0, FGR_ACT_RELU = 1, FGR_ACT_GELU_TANH = 2, FGR_ACT_SIGMOID = 3, FGR_ACT_TANH = 4,
                FGR_ACT_SILU = 5 } fgr_act;
 typedef enum { FGR_SCALE_NONE = 0, FGR_SCALE_SCALAR = 1, FGR_SCALE_PER_COLUMN = 2 } fgr_scale_kind;
-typedef enum { FGR_RED_LSE = 0, FGR_RED_SOFTMAX = 1, FGR_RED_MAXSUM = 2, FGR_RED_MAX_SUMEXP = 3 } fgr_reduce;
+typedef enum { FGR_RED_LSE = 0, FGR_RED_SOFTMAX = 1, FGR_RED_MAXSUM = 2, FGR_RED_MAX_SUMEXP = 3,
+               /* (mean, population variance) of y over N: the row statistics of a normalisation layer.  Computed
+                  per tile in two passes and merged pairwise (mean, sum of squared deviations), never as
+                  E[y^2] - E[y]^2.  Not on the FGR_PATH_SIMT_GEMV path and not in fgr_combine_shards. */
+               FGR_RED_MEANVAR = 6 } fgr_reduce;
 
 /* Execution paths (fgr_plan_info.path, fgr_desc.force_path). */
 typedef enum {
@@ -161,7 +165,7 @@ FGR_API int fgr_get_plan(const fgr_handle* h, fgr_plan_info* info /*host, out*/)
  *   bias       device fp32 [N] (or [batch, N]); NULL = no bias
  *   scale_vec  device fp32 [N]; required iff scale_kind == FGR_SCALE_PER_COLUMN
  *   Y          device, dtype, [batch, M, N]; required iff write_y or SOFTMAX
- *   out        device fp32: [batch*M] (LSE) or [batch*M, 2] (MAXSUM, MAX_SUMEXP).  SOFTMAX: optional;
+ *   out        device fp32: [batch*M] (LSE) or [batch*M, 2] (MAXSUM, MAX_SUMEXP, MEANVAR).  SOFTMAX: optional;
  *              if not NULL it receives [batch*M, 2] = (row max, sum of exp(y - max)), the statistics
  *              that P was normalised with (what fgr_combine_shards needs)
  *   workspace  device, 256-byte aligned, at least fgr_workspace_bytes(h); scratch for the
@@ -224,12 +228,12 @@ FGR_API int fgr_run_static(const fgr_desc* desc /*host*/, const void* X, const v
  * operator category "reduction" (Section 4.1, Datasets); the paper's GPU case study is a max
  * reduction over a dimension (Section 4.4.1).  The same row reductions as the fused operator,
  * applied to A itself, plus plain max and plain sum:
- *     FGR_RED_LSE, FGR_RED_MAXSUM, FGR_RED_MAX_SUMEXP, FGR_REDUCE_MAX, FGR_REDUCE_SUM -> out
+ *     FGR_RED_LSE, FGR_RED_MAXSUM, FGR_RED_MAX_SUMEXP, FGR_RED_MEANVAR, FGR_REDUCE_MAX, FGR_REDUCE_SUM -> out
  *     FGR_RED_SOFTMAX -> P[M, N] in A's dtype (P must not overlap A)
  *   A    device, dtype (fp32 or bf16), row stride lda elements (0 = N), 16-byte aligned, read once
  *        (twice for softmax, the second time normally from L2)
  *   P    device, dtype, row stride ldp (0 = N); required iff SOFTMAX
- *   out  device fp32: [M] (LSE, MAX, SUM) or [M, 2] (MAXSUM, MAX_SUMEXP); required unless SOFTMAX
+ *   out  device fp32: [M] (LSE, MAX, SUM) or [M, 2] (MAXSUM, MAX_SUMEXP, MEANVAR); required unless SOFTMAX
  * N, lda and ldp must be multiples of 8 (bf16) / 4 (fp32), else FGR_ERR_UNSUPPORTED.  One kernel
  * launch on `cuda_stream`, asynchronous, no workspace, no handle; bit-identical from run to run.
  * Rows are not split across CTAs: the kernel is bandwidth-bound once M is a few hundred or more.

@@ -17,6 +17,7 @@ FGR_F32, FGR_BF16 = 0, 1
 FGR_ACT_NONE, FGR_ACT_RELU, FGR_ACT_GELU_TANH, FGR_ACT_SIGMOID, FGR_ACT_TANH, FGR_ACT_SILU = 0, 1, 2, 3, 4, 5
 FGR_SCALE_NONE, FGR_SCALE_SCALAR, FGR_SCALE_PER_COLUMN = 0, 1, 2
 FGR_RED_LSE, FGR_RED_SOFTMAX, FGR_RED_MAXSUM, FGR_RED_MAX_SUMEXP = 0, 1, 2, 3
+FGR_RED_MEANVAR = 6
 FGR_REDUCE_MAX, FGR_REDUCE_SUM = 4, 5
 FGR_PATH_AUTO, FGR_PATH_SIMT, FGR_PATH_UMMA_TILED, FGR_PATH_UMMA_STREAM_W, FGR_PATH_SIMT_GEMV = 0, 1, 2, 3, 4
 FGR_PATH_UMMA_TF32X3 = 5

@@ -51,6 +51,15 @@ __host__ __device__ inline int part_slot(int col, int tile_n, int half_n, int sl
   return t * slots_per_tile + ((slots_per_tile == 2 && w >= half_n) ? 1 : 0);
 }
 
+// Number of matrix columns that partial slot `t` of a row covers (the last tile may be ragged).
+__host__ __device__ inline int slot_columns(int t, int N, int tile_n, int half_n, int slots_per_tile) {
+  const int tile = t / slots_per_tile, h = t - tile * slots_per_tile;
+  const int begin = tile * tile_n + (h ? half_n : 0);
+  int end = (slots_per_tile == 2 && h == 0) ? tile * tile_n + half_n : (tile + 1) * tile_n;
+  if (end > N) end = N;
+  return end > begin ? end - begin : 0;
+}
+
 // Shared-memory carve-up of the tcgen05 kernel (offsets from a 1024-byte aligned base).
 struct UmmaSmem {
   int stage_bytes, sub_bytes, x_bytes, w_bytes;   // a stage is `ksub` sub-blocks of (X tile, W tile)

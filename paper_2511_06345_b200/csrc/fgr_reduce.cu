@@ -171,12 +171,87 @@ __global__ void __launch_bounds__(kThreads, 8) reduce_rows_kernel(const ReducePa
   }
 }
 
+// (mean, population variance) of every row.  Each thread takes up to four 128-bit vectors at a time,
+// computes their mean and sum of squared deviations in registers (two passes over the registers) and
+// folds that into its running (count, mean, M2) with the pairwise update
+//   delta = mean_b - mean_a;  mean = mean_a + delta n_b / n;  M2 = M2_a + M2_b + delta^2 n_a n_b / n,
+// then the threads of a row are combined in a fixed order with the same update.  E[v^2] - E[v]^2 is
+// never formed, so a large common offset costs no accuracy.
+struct Moments { float n, mean, m2; };
+__device__ __forceinline__ Moments merge_moments(Moments a, Moments b) {
+  const float tot = a.n + b.n;
+  if (tot == 0.0f) return a;
+  const float delta = b.mean - a.mean;
+  return {tot, a.mean + delta * (b.n / tot), a.m2 + b.m2 + delta * delta * (a.n * b.n / tot)};
+}
+template <typename T, int G>
+__global__ void __launch_bounds__(kThreads, 8) meanvar_rows_kernel(const ReduceParams p) {
+  constexpr int V = Vec<T>::kElems;
+  constexpr int kRowsPerCta = kThreads / G;
+  __shared__ Moments red[kThreads / 32];
+  const int sub = threadIdx.x % G, lane = threadIdx.x & 31;
+  const long long row = (long long)blockIdx.x * kRowsPerCta + threadIdx.x / G;
+  const bool row_ok = row < p.M;
+  const T* a = static_cast<const T*>(p.A) + (row_ok ? row : 0) * p.lda;
+  Moments st = {0.0f, 0.0f, 0.0f};
+  if (row_ok) {
+    for (int c0 = sub * V; c0 < p.N; c0 += 4 * G * V) {
+      uint4 raw[4];
+      int nv = 0;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int c = c0 + u * G * V;
+        if (c < p.N) { raw[u] = *reinterpret_cast<const uint4*>(a + c); nv = u + 1; }
+      }
+      float sum = 0.0f;
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (u < nv) {
+          float v[V];
+          Vec<T>::unpack(raw[u], v);
+#pragma unroll
+          for (int j = 0; j < V; ++j) sum += v[j];
+        }
+      Moments ch = {(float)(nv * V), 0.0f, 0.0f};
+      ch.mean = sum / ch.n;
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (u < nv) {
+          float v[V];
+          Vec<T>::unpack(raw[u], v);
+#pragma unroll
+          for (int j = 0; j < V; ++j) ch.m2 = fmaf(v[j] - ch.mean, v[j] - ch.mean, ch.m2);
+        }
+      st = merge_moments(st, ch);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) {
+    Moments ot = {__shfl_xor_sync(0xffffffffu, st.n, o), __shfl_xor_sync(0xffffffffu, st.mean, o),
+                  __shfl_xor_sync(0xffffffffu, st.m2, o)};
+    st = (lane & o) ? merge_moments(ot, st) : merge_moments(st, ot);   // the lower lane's triple on the left in both
+  }
+  if (G == kThreads) {
+    if (lane == 0) red[threadIdx.x >> 5] = st;
+    __syncthreads();
+    st = red[0];
+#pragma unroll
+    for (int w = 1; w < kThreads / 32; ++w) st = merge_moments(st, red[w]);
+  }
+  if (row_ok && sub == 0) reinterpret_cast<float2*>(p.out)[row] = make_float2(st.mean, st.m2 / (float)p.N);
+}
+
 template <typename T>
 cudaError_t launch(const ReduceParams& p, cudaStream_t s) {
   const bool exp_kind = p.kind == FGR_RED_LSE || p.kind == FGR_RED_SOFTMAX || p.kind == FGR_RED_MAX_SUMEXP;
   const bool warp_rows = p.N <= 32 * Vec<T>::kElems * 8;   // a warp covers the row in at most two iterations
   const unsigned grid = warp_rows ? (unsigned)((p.M + kThreads / 32 - 1) / (kThreads / 32)) : (unsigned)p.M;
   const bool sum_kind = p.kind == FGR_RED_MAXSUM || p.kind == FGR_REDUCE_SUM;
+  if (p.kind == FGR_RED_MEANVAR) {
+    if (warp_rows) meanvar_rows_kernel<T, 32><<<grid, kThreads, 0, s>>>(p);
+    else meanvar_rows_kernel<T, kThreads><<<grid, kThreads, 0, s>>>(p);
+    return cudaGetLastError();
+  }
 #define FGR_REDUCE_LAUNCH(Gv) \
   do { \
     if (exp_kind) reduce_rows_kernel<T, Gv, true, false><<<grid, kThreads, 0, s>>>(p); \
@@ -194,7 +269,7 @@ cudaError_t launch(const ReduceParams& p, cudaStream_t s) {
 extern "C" int fgr_reduce_rows(const fgr_reduce_desc* d, const void* A, void* P, float* out, void* cuda_stream) {
   if (!d || d->struct_bytes != sizeof(fgr_reduce_desc) || !A) return FGR_ERR_INVALID_ARG;
   if (d->dtype != FGR_F32 && d->dtype != FGR_BF16) return FGR_ERR_INVALID_ARG;
-  if (d->reduce < FGR_RED_LSE || d->reduce > FGR_REDUCE_SUM) return FGR_ERR_INVALID_ARG;
+  if (d->reduce < FGR_RED_LSE || d->reduce > FGR_RED_MEANVAR) return FGR_ERR_INVALID_ARG;
   if (d->M < 1 || d->N < 1 || d->device < 0 || d->lda < 0 || d->ldp < 0) return FGR_ERR_INVALID_ARG;
   const int g = d->dtype == FGR_F32 ? 4 : 8;   // elements per 16 bytes
   const long long lda = d->lda ? d->lda : d->N, ldp = d->ldp ? d->ldp : d->N;

@@ -128,8 +128,10 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(const Params p) {
     }
   }
   T* Y = static_cast<T*>(p.Y) + (long long)bt * p.bsy;
-  const bool exp_kind = p.reduce != FGR_RED_MAXSUM;
+  const bool meanvar = p.reduce == FGR_RED_MEANVAR;
+  const bool exp_kind = p.reduce != FGR_RED_MAXSUM && !meanvar;
   const bool store_y = p.write_y && p.reduce != FGR_RED_SOFTMAX;
+  const int tile_cols = p.N - n0 < kSimtTile ? p.N - n0 : kSimtTile;   // columns of this tile inside the matrix
 
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -145,7 +147,15 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(const Params p) {
     // ---- per-tile row reduction across the 16 threads that share this row
     mx = group16_max(mx);
     float second;
-    if (exp_kind) {
+    if (meanvar) {
+      // two passes over the tile's columns of this row: mean, then squared deviations from it
+      const float mean = group16_sum(sm) / (float)tile_cols;
+      float dev = 0.0f;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) if (cols_ok) dev += (y[j] - mean) * (y[j] - mean);
+      mx = mean;
+      second = group16_sum(dev);
+    } else if (exp_kind) {
       float e[4], l = 0.0f;
 #pragma unroll
       for (int j = 0; j < 4; ++j) { e[j] = cols_ok ? expf(y[j] - mx) : 0.0f; l += e[j]; }
@@ -183,6 +193,39 @@ __global__ void __launch_bounds__(256) merge_kernel(const Params p) {
   const long long row = warp * (32 / G) + lane / G;
   const bool row_ok = row < (long long)p.batch * p.M;
   const float2* src = reinterpret_cast<const float2*>(p.parts) + (row_ok ? row : 0) * p.parts_per_row;
+  if (p.reduce == FGR_RED_MEANVAR) {
+    // pairs are (mean, sum of squared deviations) of a slot; the slot's column count follows from the
+    // tiling.  Pairwise update: delta = mean_b - mean_a; mean += delta n_b / n; M2 += M2_b + delta^2 n_a n_b / n
+    float n = 0.0f, mean = 0.0f, m2 = 0.0f;
+    for (int t = sub; t < p.parts_per_row; t += G) {
+      const float nb = (float)slot_columns(t, p.N, p.tile_n, p.half_n, p.slots_per_tile);
+      if (nb > 0.0f) {
+        const float2 v = src[t];
+        const float tot = n + nb, delta = v.x - mean;
+        mean += delta * (nb / tot);
+        m2 += v.y + delta * delta * (n * nb / tot);
+        n = tot;
+      }
+    }
+#pragma unroll
+    for (int o = G / 2; o >= 1; o >>= 1) {
+      const float on = __shfl_xor_sync(0xffffffffu, n, o), om = __shfl_xor_sync(0xffffffffu, mean, o),
+                  o2 = __shfl_xor_sync(0xffffffffu, m2, o);
+      // the lower lane's triple is always the left operand, so both lanes compute the same bits
+      const bool hi = (lane & o) != 0;
+      const float na = hi ? on : n, ma = hi ? om : mean, qa = hi ? o2 : m2;
+      const float nb = hi ? n : on, mb = hi ? mean : om, qb = hi ? m2 : o2;
+      const float tot = na + nb;
+      if (tot > 0.0f) {
+        const float delta = mb - ma;
+        mean = ma + delta * (nb / tot);
+        m2 = qa + qb + delta * delta * (na * nb / tot);
+      }
+      n = tot;
+    }
+    if (sub == 0 && row_ok) reinterpret_cast<float2*>(p.out)[row] = make_float2(mean, m2 / (float)p.N);
+    return;
+  }
   const bool exp_kind = p.reduce != FGR_RED_MAXSUM;
   float a = -CUDART_INF_F, b = 0.0f;
   for (int t = sub; t < p.parts_per_row; t += G) {

@@ -17,7 +17,7 @@ cudaError_t umma_prepare(int) {
 cudaError_t launch_umma(const Params& p, const void* tmap_x, const void* tmap_w, int grid, int smem_bytes,
                         cudaStream_t stream) {
   const bool softmax = p.reduce == FGR_RED_SOFTMAX;
-  const bool exp_kind = p.reduce != FGR_RED_MAXSUM;
+  const bool exp_kind = p.reduce == FGR_RED_LSE || p.reduce == FGR_RED_SOFTMAX || p.reduce == FGR_RED_MAX_SUMEXP;
   const bool wy = p.write_y && !softmax;
   // exp kinds that do not store y fold log2(e) into the staged scale vector, so they always multiply
   const bool sc = (exp_kind && !wy) || p.scale_kind != FGR_SCALE_NONE;

@@ -290,7 +290,8 @@ __device__ __forceinline__ TileCoord tile_coord(long long t, const Params& p, in
 //   RED : fgr_reduce       WY : store y as bf16 (ignored for softmax, which always stores)
 template <int ACT, bool SC, int RED, bool WY>
 struct Variant {
-  static constexpr bool kExp = RED != FGR_RED_MAXSUM;
+  static constexpr bool kExp = RED == FGR_RED_LSE || RED == FGR_RED_SOFTMAX || RED == FGR_RED_MAX_SUMEXP;
+  static constexpr bool kMeanVar = RED == FGR_RED_MEANVAR;
   static constexpr bool kSoftmax = RED == FGR_RED_SOFTMAX;
   static constexpr bool kStoreY = WY && !kSoftmax;
   // exp kinds work in log2 units; when y itself is not stored the factor log2(e) is folded into
@@ -647,6 +648,23 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
           }
           if (row_ok) store16(cc, yy, nv);
         });
+      } else if constexpr (V::kMeanVar) {
+        // pass A: sum of this warp's columns (and the Y store); pass B: squared deviations from their mean
+        sweep([&](float* yy, int cc, int nv) {
+          if constexpr (V::kStoreY) {
+            if (row_ok) store16(cc, yy, nv);
+          }
+#pragma unroll
+          for (int j = 0; j < kChunk; ++j) if (real(j, nv)) r1 += yy[j];
+        });
+        const float mean = c_lim > c_begin ? r1 / (float)(c_lim - c_begin) : 0.0f;
+        float dev = 0.0f;
+        sweep([&](float* yy, int, int nv) {
+#pragma unroll
+          for (int j = 0; j < kChunk; ++j) if (real(j, nv)) dev = fmaf(yy[j] - mean, yy[j] - mean, dev);
+        });
+        r0 = mean;
+        r1 = dev;
       } else {
         sweep([&](float* yy, int cc, int nv) {
           if constexpr (V::kStoreY) {
@@ -743,7 +761,9 @@ cudaError_t prepare_one() {
   X(false, FGR_RED_MAXSUM, false) X(false, FGR_RED_MAXSUM, true) X(true, FGR_RED_MAXSUM, false)   \
   X(true, FGR_RED_MAXSUM, true) X(true, FGR_RED_LSE, false) X(false, FGR_RED_LSE, true)           \
   X(true, FGR_RED_LSE, true) X(true, FGR_RED_MAX_SUMEXP, false) X(false, FGR_RED_MAX_SUMEXP, true) \
-  X(true, FGR_RED_MAX_SUMEXP, true) X(true, FGR_RED_SOFTMAX, false)
+  X(true, FGR_RED_MAX_SUMEXP, true) X(true, FGR_RED_SOFTMAX, false)                               \
+  X(false, FGR_RED_MEANVAR, false) X(false, FGR_RED_MEANVAR, true) X(true, FGR_RED_MEANVAR, false) \
+  X(true, FGR_RED_MEANVAR, true)
 
 template <int ACT>
 cudaError_t launch_act(bool sc, int red, bool wy, const Params& p, const CUtensorMap& tx, const CUtensorMap& tw, int grid,
