@@ -171,19 +171,12 @@ __global__ void __launch_bounds__(kThreads, 8) reduce_rows_kernel(const ReducePa
   }
 }
 
-// (mean, population variance) of every row.  Each thread takes up to four 128-bit vectors at a time,
-// computes their mean and sum of squared deviations in registers (two passes over the registers) and
-// folds that into its running (count, mean, M2) with the pairwise update
-//   delta = mean_b - mean_a;  mean = mean_a + delta n_b / n;  M2 = M2_a + M2_b + delta^2 n_a n_b / n,
-// then the threads of a row are combined in a fixed order with the same update.  E[v^2] - E[v]^2 is
-// never formed, so a large common offset costs no accuracy.
+// (mean, population variance) of every row.  Each thread accumulates sum (v - c) and sum (v - c)^2
+// over its elements, c being the first element it sees (a shift inside the data's range, so the
+// final  M2 = sum d^2 - (sum d)^2 / n  cancels only mildly; E[v^2] - E[v]^2 of the raw values is never
+// formed and a large common offset costs no accuracy).  Four instructions per element and no
+// division in the loop.  The threads of a row are then combined by fixed shuffle / shared-memory sums.
 struct Moments { float n, mean, m2; };
-__device__ __forceinline__ Moments merge_moments(Moments a, Moments b) {
-  const float tot = a.n + b.n;
-  if (tot == 0.0f) return a;
-  const float delta = b.mean - a.mean;
-  return {tot, a.mean + delta * (b.n / tot), a.m2 + b.m2 + delta * delta * (a.n * b.n / tot)};
-}
 template <typename T, int G>
 __global__ void __launch_bounds__(kThreads, 8) meanvar_rows_kernel(const ReduceParams p) {
   constexpr int V = Vec<T>::kElems;
@@ -194,7 +187,9 @@ __global__ void __launch_bounds__(kThreads, 8) meanvar_rows_kernel(const ReduceP
   const bool row_ok = row < p.M;
   const T* a = static_cast<const T*>(p.A) + (row_ok ? row : 0) * p.lda;
   Moments st = {0.0f, 0.0f, 0.0f};
-  if (row_ok) {
+  if (row_ok && sub * V < p.N) {
+    float shift = 0.0f, s1 = 0.0f, s2 = 0.0f;
+    int cnt = 0;
     for (int c0 = sub * V; c0 < p.N; c0 += 4 * G * V) {
       uint4 raw[4];
       int nv = 0;
@@ -203,41 +198,45 @@ __global__ void __launch_bounds__(kThreads, 8) meanvar_rows_kernel(const ReduceP
         const int c = c0 + u * G * V;
         if (c < p.N) { raw[u] = *reinterpret_cast<const uint4*>(a + c); nv = u + 1; }
       }
-      float sum = 0.0f;
+      if (cnt == 0) shift = __uint_as_float(sizeof(T) == 4 ? raw[0].x : raw[0].x << 16);   // the thread's first element
 #pragma unroll
       for (int u = 0; u < 4; ++u)
         if (u < nv) {
           float v[V];
           Vec<T>::unpack(raw[u], v);
 #pragma unroll
-          for (int j = 0; j < V; ++j) sum += v[j];
+          for (int j = 0; j < V; ++j) { const float d = v[j] - shift; s1 += d; s2 = fmaf(d, d, s2); }
         }
-      Moments ch = {(float)(nv * V), 0.0f, 0.0f};
-      ch.mean = sum / ch.n;
-#pragma unroll
-      for (int u = 0; u < 4; ++u)
-        if (u < nv) {
-          float v[V];
-          Vec<T>::unpack(raw[u], v);
-#pragma unroll
-          for (int j = 0; j < V; ++j) ch.m2 = fmaf(v[j] - ch.mean, v[j] - ch.mean, ch.m2);
-        }
-      st = merge_moments(st, ch);
+      cnt += nv * V;
     }
+    st.n = (float)cnt;
+    const float md = s1 / st.n;
+    st.mean = shift + md;
+    st.m2 = fmaxf(s2 - s1 * md, 0.0f);
   }
-#pragma unroll
-  for (int o = 16; o >= 1; o >>= 1) {
-    Moments ot = {__shfl_xor_sync(0xffffffffu, st.n, o), __shfl_xor_sync(0xffffffffu, st.mean, o),
-                  __shfl_xor_sync(0xffffffffu, st.m2, o)};
-    st = (lane & o) ? merge_moments(ot, st) : merge_moments(st, ot);   // the lower lane's triple on the left in both
-  }
+  // Combine the threads of a row without a chain of pairwise updates: the row mean is the count-
+  // weighted mean of the thread means, and by the parallel-axis identity
+  //   M2 = sum_i [ M2_i + n_i (mean_i - mean)^2 ]   (all terms non-negative: nothing cancels).
+  float cn = warp_sum(st.n), cs = warp_sum(st.n * st.mean);
   if (G == kThreads) {
-    if (lane == 0) red[threadIdx.x >> 5] = st;
+    if (lane == 0) red[threadIdx.x >> 5] = {cn, cs, 0.0f};
     __syncthreads();
-    st = red[0];
+    cn = 0.0f; cs = 0.0f;
 #pragma unroll
-    for (int w = 1; w < kThreads / 32; ++w) st = merge_moments(st, red[w]);
+    for (int w = 0; w < kThreads / 32; ++w) { cn += red[w].n; cs += red[w].mean; }
   }
+  const float mean = cn > 0.0f ? cs / cn : 0.0f;
+  const float dm = st.mean - mean;
+  float q = warp_sum(fmaf(st.n * dm, dm, st.m2));
+  if (G == kThreads) {
+    if (lane == 0) red[threadIdx.x >> 5].m2 = q;
+    __syncthreads();
+    q = 0.0f;
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) q += red[w].m2;
+  }
+  st.mean = mean;
+  st.m2 = q;
   if (row_ok && sub == 0) reinterpret_cast<float2*>(p.out)[row] = make_float2(st.mean, st.m2 / (float)p.N);
 }
 

@@ -88,6 +88,6 @@ def test_reduce_rows_deterministic_and_argument_checks(cuda_device):
     assert f(4, 12, fgr.FGR_BF16, fgr.FGR_RED_LSE, x, None, x) == fgr.FGR_ERR_UNSUPPORTED      # N % 8
     assert f(4, 16, fgr.FGR_BF16, fgr.FGR_RED_LSE, x, None, None) == fgr.FGR_ERR_INVALID_ARG    # out missing
     assert f(4, 16, fgr.FGR_BF16, fgr.FGR_RED_SOFTMAX, x, None, x) == fgr.FGR_ERR_INVALID_ARG   # P missing
-    assert f(4, 16, fgr.FGR_BF16, 6, x, None, x) == fgr.FGR_ERR_INVALID_ARG
+    assert f(4, 16, fgr.FGR_BF16, 7, x, None, x) == fgr.FGR_ERR_INVALID_ARG
     assert f(4, 16, fgr.FGR_BF16, fgr.FGR_RED_LSE, x, None, x, lda=8) == fgr.FGR_ERR_INVALID_ARG
     assert f(4, 16, fgr.FGR_BF16, fgr.FGR_RED_LSE, x.data_ptr() + 4, None, x) == fgr.FGR_ERR_INVALID_ARG
