@@ -46,7 +46,7 @@ constexpr int kDefaultSms = 148;
 // core truncates its fp32 accumulator once per instruction (measured: a relative bias of about 7e-9 per
 // unit of K, towards zero); 128 keeps that below 1e-6, the level of an fp32 FMA loop at K of a few thousand.
 constexpr int kTf32ChunkBlocks = 4;
-constexpr double kTf32MinFlop = 4.0e9;   // below this the fp32 problem stays on the CUDA-core path
+constexpr double kTf32MinFlop = 1.0e9;   // below this the fp32 problem stays on the CUDA-core path (measured: the two cross near 512^3)
 size_t align256(size_t x) { return (x + 255u) & ~(size_t)255u; }
 
 int elem_bytes(int dtype) { return dtype == FGR_F32 ? 4 : 2; }
