@@ -85,3 +85,38 @@ def test_c5_batched_sampled_rows(cuda_device, reduce):
     pw = gi.make_config("c5", write_y=1, batch=4)
     Y, out, _ = run_gpu(pw)
     compare(pw, Y, out, rows=_rows(pw.batch * pw.M, 1024, 16, 7))
+
+
+def test_f2_fp32_tensor_core_sampled_rows(cuda_device):
+    """The benchmark's fp32 workload (c2's shapes and epilogue in fp32: the 3xTF32 path) at full size."""
+    from test_tf32x3 import _slack
+    p = gi.make_config("c2", dtype=gi.DTYPE_F32)
+    Y, out, plan = run_gpu(p)
+    assert plan["path"] == fgr.FGR_PATH_UMMA_TF32X3 and plan["cta_pair"] == 2 and plan["tile_n"] == 256
+    rows = _rows(p.M, 128, 24, 8)
+    ys, os_, yr = _slack(p, rows)
+    w = compare(p, Y, out, rows=rows, tcgen05=False, y_slack=ys, out_slack=os_, y_rel_slack=yr)
+    assert w["Y"] <= 1e-4 and w["out"] <= 1e-4
+    assert (out[:, 0] >= 0).all() and (out[:, 1] >= out[:, 0] - 1e-4).all()
+
+
+def test_v2_convolution_sampled_rows(cuda_device):
+    """The benchmark's convolution workload at full size: 8 signals of 2051 x 512 channels, 4096 shared
+    filters of 4 taps, c2's epilogue."""
+    p = gi.make_config("c2", batch=8, M=2048, N=4096, K=2048, conv_taps=4, w_shared=1)
+    assert p.X.shape == (8, 2051, 512) and p.W.shape == (1, 4096, 2048)
+    Y, out, plan = run_gpu(p)
+    assert plan["path"] == fgr.FGR_PATH_UMMA_TILED and plan["num_tiles"] == 1024
+    rows = _rows(p.batch * p.M, 2048, 32, 9)
+    import copy
+    import oracle
+    # the oracle's window matrix for the sampled rows only (the full one would be 8 x 2048 x 2048)
+    q = copy.copy(p)
+    q.conv_taps, q.batch, q.M = 0, 1, len(rows)
+    q.X = np.stack([p.X[r // p.M, (r % p.M):(r % p.M) + 4, :].reshape(-1) for r in rows])[None]
+    q.W = p.W
+    Yr, outr, _ = oracle.run_problem(q)
+    got_y, got_o = Y[rows], out[rows]
+    assert (np.abs(got_y - Yr) <= 4.5e-3 * np.abs(Yr) + 2e-5 * (1 + np.abs(Yr).max())).all()
+    assert (np.abs(got_o - outr) <= 2e-4 * (1 + np.abs(outr)) + 1e-6 * np.abs(Yr).sum(1, keepdims=True)).all()
+    assert (np.abs(got_y - Yr) / (1 + np.abs(Yr))).max() <= 2e-2
