@@ -72,7 +72,12 @@ def test_forced_tiles_and_paths():
     p = _plan(1, 300, 520, 200, fgr.FGR_BF16, 0, 0, 0, force_path=fgr.FGR_PATH_UMMA_TILED, force_tile_n=112)
     assert p.tile_n == 112 and p.parts_per_row == 2 * 5 and p.num_tiles == 3 * 5
     p = _plan(1, 300, 520, 200, fgr.FGR_BF16, 0, 0, 0, force_path=fgr.FGR_PATH_UMMA_TILED, force_cta_pair=1)
-    assert p.cta_pair == 1 and p.tile_m == 128 and p.num_tiles == 3 * 3 and p.stages == 4
+    # 9 tiles of 256 columns would leave most SMs idle: the tiles are narrowed until one wave fills more of them
+    assert p.cta_pair == 1 and p.tile_m == 128 and p.tile_n == 32 and p.num_tiles == 3 * 17
+    p = _plan(1, 300, 520, 200, fgr.FGR_BF16, 0, 0, 0, force_path=fgr.FGR_PATH_UMMA_TILED, force_cta_pair=1, force_tile_n=256)
+    assert p.num_tiles == 3 * 3 and p.stages == 4
+    mid = _plan(1, 256, 8192, 4096, fgr.FGR_BF16, 0, 0, 0)
+    assert mid.path == fgr.FGR_PATH_UMMA_TILED and (mid.tile_n, mid.cta_pair, mid.num_tiles) == (128, 2, 64)
     p = _plan(1, 300, 520, 200, fgr.FGR_BF16, 0, 0, 0, force_path=fgr.FGR_PATH_UMMA_TILED, force_cta_pair=2, force_tile_n=64)
     assert p.cta_pair == 2 and p.tile_m == 256 and p.num_tiles == 2 * 9 and p.grid == 36
     with pytest.raises(fgr.FgrError):
