@@ -102,14 +102,28 @@ __global__ void __launch_bounds__(kThreads, 8) reduce_rows_kernel(const ReducePa
         if (c < p.N) { raw[u] = *reinterpret_cast<const uint4*>(a + c); nv = u + 1; }
       }
       float vm = -CUDART_INF_F;
+      if constexpr (sizeof(T) == 2 && !SUM) {
+        // maximum of the packed pairs first (one instruction per two elements), unpacked once at the end
+        __nv_bfloat162 m2 = *reinterpret_cast<const __nv_bfloat162*>(&raw[0].x);
 #pragma unroll
-      for (int u = 0; u < 4; ++u)
-        if (u < nv) {
-          float v[V];
-          Vec<T>::unpack(raw[u], v);
+        for (int u = 0; u < 4; ++u)
+          if (u < nv) {
+            const uint32_t w[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
 #pragma unroll
-          for (int j = 0; j < V; ++j) { vm = fmaxf(vm, v[j]); if (SUM) st.s += v[j]; }
-        }
+            for (int i = 0; i < 4; ++i) m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162*>(&w[i]));
+          }
+        const uint32_t mb = *reinterpret_cast<const uint32_t*>(&m2);
+        vm = fmaxf(__uint_as_float(mb << 16), __uint_as_float(mb & 0xffff0000u));
+      } else {
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (u < nv) {
+            float v[V];
+            Vec<T>::unpack(raw[u], v);
+#pragma unroll
+            for (int j = 0; j < V; ++j) { vm = fmaxf(vm, v[j]); if (SUM) st.s += v[j]; }
+          }
+      }
       if (EXP) {
         const float mn = fmaxf(st.m, vm);
         const float off = mn * kLog2e;
@@ -135,6 +149,7 @@ __global__ void __launch_bounds__(kThreads, 8) reduce_rows_kernel(const ReducePa
   if (G == kThreads) {
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = st;
     __syncthreads();
+    if (p.kind != FGR_RED_SOFTMAX && threadIdx.x != 0) return;   // only softmax needs the row's pair in every thread
     float m = red[0].m;
 #pragma unroll
     for (int w = 1; w < kThreads / 32; ++w) m = fmaxf(m, red[w].m);
@@ -214,30 +229,34 @@ __global__ void __launch_bounds__(kThreads, 8) meanvar_rows_kernel(const ReduceP
     st.mean = shift + md;
     st.m2 = fmaxf(s2 - s1 * md, 0.0f);
   }
-  // Combine the threads of a row without a chain of pairwise updates: the row mean is the count-
+  // Combine the threads of a warp without a chain of pairwise updates: the warp mean is the count-
   // weighted mean of the thread means, and by the parallel-axis identity
   //   M2 = sum_i [ M2_i + n_i (mean_i - mean)^2 ]   (all terms non-negative: nothing cancels).
-  float cn = warp_sum(st.n), cs = warp_sum(st.n * st.mean);
+  const float cn = warp_sum(st.n), cs = warp_sum(st.n * st.mean);
+  const float wmean = cn > 0.0f ? cs / cn : 0.0f;
+  const float dm = st.mean - wmean;
+  const float q = warp_sum(fmaf(st.n * dm, dm, st.m2));
+  Moments row_m = {cn, wmean, q};
   if (G == kThreads) {
-    if (lane == 0) red[threadIdx.x >> 5] = {cn, cs, 0.0f};
+    // a row spread over the CTA: thread 0 folds the eight warp triples, in warp order, with the pairwise update
+    //   delta = mean_b - mean_a;  mean = mean_a + delta n_b / n;  M2 = M2_a + M2_b + delta^2 n_a n_b / n
+    if (lane == 0) red[threadIdx.x >> 5] = row_m;
     __syncthreads();
-    cn = 0.0f; cs = 0.0f;
+    if (threadIdx.x != 0) return;
+    row_m = red[0];
 #pragma unroll
-    for (int w = 0; w < kThreads / 32; ++w) { cn += red[w].n; cs += red[w].mean; }
+    for (int w = 1; w < kThreads / 32; ++w) {
+      const Moments b = red[w];
+      const float tot = row_m.n + b.n;
+      if (tot > 0.0f) {
+        const float delta = b.mean - row_m.mean, wb = b.n / tot;
+        row_m.m2 = row_m.m2 + b.m2 + delta * delta * (row_m.n * wb);
+        row_m.mean = fmaf(delta, wb, row_m.mean);
+        row_m.n = tot;
+      }
+    }
   }
-  const float mean = cn > 0.0f ? cs / cn : 0.0f;
-  const float dm = st.mean - mean;
-  float q = warp_sum(fmaf(st.n * dm, dm, st.m2));
-  if (G == kThreads) {
-    if (lane == 0) red[threadIdx.x >> 5].m2 = q;
-    __syncthreads();
-    q = 0.0f;
-#pragma unroll
-    for (int w = 0; w < kThreads / 32; ++w) q += red[w].m2;
-  }
-  st.mean = mean;
-  st.m2 = q;
-  if (row_ok && sub == 0) reinterpret_cast<float2*>(p.out)[row] = make_float2(st.mean, st.m2 / (float)p.N);
+  if (row_ok && sub == 0) reinterpret_cast<float2*>(p.out)[row] = make_float2(row_m.mean, row_m.m2 / (float)p.N);
 }
 
 template <typename T>
