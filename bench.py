@@ -376,6 +376,9 @@ REDUCE_CONFIGS = {   # stand-alone row reduction of a bf16 matrix, the paper's G
     "r_lse": dict(M=8192, N=8192, kind=0, name="lse"),
     "r_softmax": dict(M=8192, N=8192, kind=1, name="softmax"),
     "r_meanvar": dict(M=8192, N=8192, kind=6, name="meanvar"),
+    # few, long rows (the shape of a reduction over a flattened dimension): clusters of 8 CTAs share a row
+    "r_lse_long": dict(M=16, N=4194304, kind=0, name="lse"),
+    "r_max_long": dict(M=16, N=4194304, kind=4, name="max"),
 }
 
 

@@ -236,7 +236,9 @@ FGR_API int fgr_run_static(const fgr_desc* desc /*host*/, const void* X, const v
  *   out  device fp32: [M] (LSE, MAX, SUM) or [M, 2] (MAXSUM, MAX_SUMEXP, MEANVAR); required unless SOFTMAX
  * N, lda and ldp must be multiples of 8 (bf16) / 4 (fp32), else FGR_ERR_UNSUPPORTED.  One kernel
  * launch on `cuda_stream`, asynchronous, no workspace, no handle; bit-identical from run to run.
- * Rows are not split across CTAs: the kernel is bandwidth-bound once M is a few hundred or more.
+ * A row is reduced by a warp (short rows), a CTA, or - when there are fewer than about 300 rows and they
+ * are long - by a thread-block cluster of 2, 4 or 8 CTAs whose per-CTA results are combined through
+ * distributed shared memory (no scratch memory, still one launch).  MEANVAR rows always take one CTA.
  */
 enum { FGR_REDUCE_MAX = 4, FGR_REDUCE_SUM = 5 };   /* further values of `reduce` for fgr_reduce_rows only */
 typedef struct fgr_reduce_desc {

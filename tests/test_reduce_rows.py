@@ -91,3 +91,26 @@ def test_reduce_rows_deterministic_and_argument_checks(cuda_device):
     assert f(4, 16, fgr.FGR_BF16, 7, x, None, x) == fgr.FGR_ERR_INVALID_ARG
     assert f(4, 16, fgr.FGR_BF16, fgr.FGR_RED_LSE, x, None, x, lda=8) == fgr.FGR_ERR_INVALID_ARG
     assert f(4, 16, fgr.FGR_BF16, fgr.FGR_RED_LSE, x.data_ptr() + 4, None, x) == fgr.FGR_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("dtype", [gi.DTYPE_F32, gi.DTYPE_BF16])
+@pytest.mark.parametrize("kind", KINDS)
+@pytest.mark.parametrize("shape", [(1, 1048576), (16, 262144), (5, 100008), (2, 33000), (40, 65536 + 8)])
+def test_reduce_rows_few_long_rows_cluster(cuda_device, dtype, kind, shape):
+    """Few, long rows: a cluster of 2, 4 or 8 CTAs shares a row and the per-CTA states are combined
+    through distributed shared memory (ragged segments included)."""
+    M, N = shape
+    _check(_matrix(M, N, dtype, seed=60 + M, std=3.0), N, dtype, kind)
+
+
+def test_reduce_rows_cluster_deterministic_and_dominant_segment(cuda_device):
+    a = _matrix(4, 524288, gi.DTYPE_BF16, seed=77)
+    r = [_run(a, 524288, gi.DTYPE_BF16, fgr.FGR_RED_LSE)[1] for _ in range(3)]
+    assert np.array_equal(r[0], r[1]) and np.array_equal(r[0], r[2])
+    # the row maximum, by a wide margin, in the last CTA's segment only: the other states rescale to zero
+    f = gi.normal(78, 9, 4 * 524288, 1.0).reshape(4, 524288)
+    f[:, -5] = 300.0
+    for dtype in (gi.DTYPE_F32, gi.DTYPE_BF16):
+        a = f if dtype == gi.DTYPE_F32 else gi.f32_to_bf16_bits(f).reshape(f.shape)
+        _check(a, 524288, dtype, fgr.FGR_RED_LSE)
+        _check(a, 524288, dtype, fgr.FGR_RED_SOFTMAX)
