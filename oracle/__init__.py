@@ -52,6 +52,9 @@ def lib() -> ctypes.CDLL:
         _lib.fgr_oracle_rows.restype = ctypes.c_int
         _lib.fgr_oracle_rows.argtypes = [ctypes.POINTER(_Problem)] + [ctypes.c_void_p] * 5 + [
             ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int]
+        _lib.fgr_oracle_rows_residual.restype = ctypes.c_int
+        _lib.fgr_oracle_rows_residual.argtypes = [ctypes.POINTER(_Problem)] + [ctypes.c_void_p] * 6 + [
+            ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int]
         _lib.fgr_oracle_reduce_rows.restype = ctypes.c_int
         _lib.fgr_oracle_reduce_rows.argtypes = [ctypes.c_int32] * 4 + [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
                                                 ctypes.c_void_p]
@@ -79,7 +82,7 @@ def _ptr(a):
 
 
 def run(X, W, bias, scale_vec, *, dtype, act, scale_kind, reduce, scale=1.0, bias_per_batch=0,
-        rows=None, want_y=True, nthreads=0):
+        rows=None, want_y=True, nthreads=0, residual=None):
     """Evaluates the operator's definition in fp64.
 
     X [batch, M, K] and W [batch, N, K] (2-D arrays are taken as batch 1; a W of batch 1 is used for
@@ -87,6 +90,8 @@ def run(X, W, bias, scale_vec, *, dtype, act, scale_kind, reduce, scale=1.0, bia
     (``dtype == F32``) or uint16 bf16 bit patterns (``dtype == BF16``).  ``bias`` fp32 [N]
     (or [batch, N] with ``bias_per_batch``) or None; ``scale_vec`` fp32 [N] or None.
     ``rows``: global row indices (bt * M + m) to evaluate; None = all rows.
+    ``residual``: R [batch, M, N] in the dtype of X (fp32 values or bf16 bit patterns), added to y
+    after the scale, or None.
 
     Returns ``(Y, out, threads)``: Y fp64 [nrows, N] (y, or P for SOFTMAX; None unless
     ``want_y``), out fp64 [nrows, width] (None for SOFTMAX), threads used.
@@ -124,6 +129,15 @@ def run(X, W, bias, scale_vec, *, dtype, act, scale_kind, reduce, scale=1.0, bia
     Y = np.empty((nrows, N), dtype=np.float64) if need_y else None
     out = np.empty((nrows, w), dtype=np.float64) if w else None
     prob = _Problem(batch, M, N, K, dtype, act, scale_kind, reduce, float(scale), int(bias_per_batch), 0)
+    if residual is not None:
+        residual = np.ascontiguousarray(residual)
+        if residual.dtype != want or residual.size != batch * M * N:
+            raise TypeError("residual must be %s [batch, M, N]" % want.__name__)
+        rc = lib().fgr_oracle_rows_residual(ctypes.byref(prob), _ptr(X), _ptr(W), _ptr(bias), _ptr(scale_vec),
+                                            _ptr(residual), _ptr(rows_arr), nrows, _ptr(Y), _ptr(out), int(nthreads))
+        if rc < 0:
+            raise ValueError("fgr_oracle_rows_residual rejected its arguments (code %d)" % rc)
+        return Y, out, rc
     rc = lib().fgr_oracle_rows(ctypes.byref(prob), _ptr(X), _ptr(W), _ptr(bias), _ptr(scale_vec), _ptr(rows_arr),
                                nrows, _ptr(Y), _ptr(out), int(nthreads))
     if rc < 0:
@@ -166,10 +180,10 @@ def run_problem(p, rows=None, want_y=True, nthreads=0):
     if getattr(p, "conv_taps", 0) > 1:
         return run(conv1d_windows(p.X, p.conv_taps), p.W, p.bias, p.scale_vec, dtype=p.dtype, act=p.act,
                    scale_kind=p.scale_kind, reduce=p.reduce, scale=p.scale, bias_per_batch=p.bias_per_batch,
-                   rows=rows, want_y=want_y, nthreads=nthreads)
+                   rows=rows, want_y=want_y, nthreads=nthreads, residual=getattr(p, "residual", None))
     return run(p.X, p.W, p.bias, p.scale_vec, dtype=p.dtype, act=p.act, scale_kind=p.scale_kind,
                reduce=p.reduce, scale=p.scale, bias_per_batch=p.bias_per_batch, rows=rows, want_y=want_y,
-               nthreads=nthreads)
+               nthreads=nthreads, residual=getattr(p, "residual", None))
 
 
 def reduce_rows(A, *, dtype, kind):

@@ -16,7 +16,8 @@
  * reduction over the last dimension), written as three nested loops in fp64:
  *
  *   z[m,n] = sum_{k = 0 .. K-1, ascending} X[m,k] * W[n,k]
- *   y[m,n] = act(z[m,n] + b[n]) * s[n]
+ *   y[m,n] = act(z[m,n] + b[n]) * s[n]  ( + R[m,n] when a residual tensor is given: a skip connection
+ *            added after the scale; the reductions then run over this y )
  *   mx[m]  = max_n y[m,n]
  *   LSE        : out[m]   = mx + log( sum_n exp(y - mx) )
  *   SOFTMAX    : P[m,n]   = exp(y - mx) / sum_n exp(y - mx)
@@ -93,7 +94,7 @@ double fgr_oracle_act(int act, double u) {
 /* One row: fills y[0..N) and, when red != NULL, the reduction (1 or 2 values);
  * for SOFTMAX y is overwritten by P. */
 static void oracle_row(const fgr_oracle_problem* p, const void* X, const void* W, const float* bias,
-                       const float* scale_vec, int64_t bt, int64_t m, double* y, double* red) {
+                       const float* scale_vec, const void* R, int64_t bt, int64_t m, double* y, double* red) {
   const int64_t N = p->N, K = p->K, M = p->M;
   const int64_t xoff = (bt * M + m) * K;
   const int64_t woff = bt * N * K;
@@ -107,6 +108,7 @@ static void oracle_row(const fgr_oracle_problem* p, const void* X, const void* W
     if (p->scale_kind == ORC_SCALE_SCALAR) s = p->scale;
     else if (p->scale_kind == ORC_SCALE_PER_COLUMN) s = (double)scale_vec[n];
     y[n] = a * s;
+    if (R) y[n] += load_elem(R, p->dtype, (bt * M + m) * N + n);
   }
   if (p->reduce == ORC_RED_MEANVAR) {
     double sum = 0.0, dev = 0.0;
@@ -143,9 +145,9 @@ static int out_width(int reduce) {
  *   nthreads  : threads over rows (<= 0: the OpenMP default)
  * Returns the number of threads used, or a negative value on a bad argument.
  */
-int fgr_oracle_rows(const fgr_oracle_problem* p, const void* X, const void* W, const float* bias,
-                    const float* scale_vec, const int64_t* rows, int64_t nrows, double* Y, double* out,
-                    int nthreads) {
+static int oracle_rows(const fgr_oracle_problem* p, const void* X, const void* W, const float* bias,
+                       const float* scale_vec, const void* R, const int64_t* rows, int64_t nrows, double* Y, double* out,
+                       int nthreads) {
   if (!p || !X || !W || nrows < 0) return -1;
   if (p->batch < 1 || p->M < 1 || p->N < 1 || p->K < 1) return -2;
   if (p->dtype != ORC_F32 && p->dtype != ORC_BF16) return -3;
@@ -173,12 +175,25 @@ int fgr_oracle_rows(const fgr_oracle_problem* p, const void* X, const void* W, c
       int64_t r = rows ? rows[i] : i;
       double red[2] = {0.0, 0.0};
       double* y = Y ? Y + i * (int64_t)p->N : ybuf;
-      oracle_row(p, X, W, bias, scale_vec, r / p->M, r % p->M, y, red);
+      oracle_row(p, X, W, bias, scale_vec, R, r / p->M, r % p->M, y, red);
       if (out) for (int j = 0; j < w; ++j) out[i * w + j] = red[j];
     }
     free(ybuf);
   }
   return used;
+}
+
+int fgr_oracle_rows(const fgr_oracle_problem* p, const void* X, const void* W, const float* bias,
+                    const float* scale_vec, const int64_t* rows, int64_t nrows, double* Y, double* out,
+                    int nthreads) {
+  return oracle_rows(p, X, W, bias, scale_vec, NULL, rows, nrows, Y, out, nthreads);
+}
+
+/* The same with a residual tensor R [batch, M, N] (packed, in the dtype of X and W), added to y after the scale. */
+int fgr_oracle_rows_residual(const fgr_oracle_problem* p, const void* X, const void* W, const float* bias,
+                             const float* scale_vec, const void* R, const int64_t* rows, int64_t nrows, double* Y,
+                             double* out, int nthreads) {
+  return oracle_rows(p, X, W, bias, scale_vec, R, rows, nrows, Y, out, nthreads);
 }
 
 int fgr_oracle_out_width(int reduce) { return out_width(reduce); }

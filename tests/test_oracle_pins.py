@@ -487,3 +487,35 @@ def test_meanvar_merge_of_slices_is_exact_identity():
             n = tot
         np.testing.assert_allclose(mean, whole[:, 0], rtol=1e-13)
         np.testing.assert_allclose(M2 / n, whole[:, 1], rtol=1e-12)
+
+
+# ---------------------------------------------------------------- residual (skip connection)
+def test_residual_closed_forms_and_library():
+    X, W, b = _rand((6, 10), 71), _rand((14, 10), 71, tid=8), gi.uniform(71, 3, 14, -1, 1)
+    R = _rand((6, 14), 72, tid=5, std=3.0)
+    # W = 0: y = act(b) * s + R exactly
+    Y, out, _ = oracle.run(X, np.zeros_like(W), b, None, dtype=oracle.F32, act=oracle.ACT_RELU, scale_kind=oracle.SCALE_SCALAR,
+                           scale=2.0, reduce=oracle.RED_MAXSUM, residual=R)
+    want = np.maximum(b.astype(np.float64), 0) * 2.0 + R.astype(np.float64)
+    np.testing.assert_allclose(Y, want, rtol=0, atol=1e-15)
+    np.testing.assert_allclose(out, np.stack([want.max(1), want.sum(1)], 1), rtol=1e-15)
+    # the residual is added AFTER activation and scale (not inside the activation): library chain in fp64
+    Y, out, _ = oracle.run(X, W, b, None, dtype=oracle.F32, act=oracle.ACT_GELU_TANH, scale_kind=oracle.SCALE_SCALAR, scale=-0.5,
+                           reduce=oracle.RED_LSE, residual=R)
+    y = torch.nn.functional.gelu(torch.from_numpy(X).double() @ torch.from_numpy(W).double().T + torch.from_numpy(b).double(),
+                                 approximate="tanh") * -0.5 + torch.from_numpy(R).double()
+    np.testing.assert_allclose(Y, y.numpy(), rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(out[:, 0], torch.logsumexp(y, 1).numpy(), rtol=1e-13)
+    # a zero residual changes nothing; rows can be sampled; bf16 residual bits are widened exactly
+    Y0, out0, _ = oracle.run(X, W, b, None, dtype=oracle.F32, act=oracle.ACT_NONE, scale_kind=oracle.SCALE_NONE, reduce=oracle.RED_SOFTMAX)
+    Y1, _, _ = oracle.run(X, W, b, None, dtype=oracle.F32, act=oracle.ACT_NONE, scale_kind=oracle.SCALE_NONE, reduce=oracle.RED_SOFTMAX,
+                          residual=np.zeros_like(R))
+    np.testing.assert_array_equal(Y0, Y1)
+    Ys, _, _ = oracle.run(X, W, b, None, dtype=oracle.F32, act=oracle.ACT_NONE, scale_kind=oracle.SCALE_NONE, reduce=oracle.RED_MAXSUM,
+                          residual=R, rows=[4, 1])
+    Yf, _, _ = oracle.run(X, W, b, None, dtype=oracle.F32, act=oracle.ACT_NONE, scale_kind=oracle.SCALE_NONE, reduce=oracle.RED_MAXSUM, residual=R)
+    np.testing.assert_array_equal(Ys, Yf[[4, 1]])
+    Xb, Wb, Rb = gi.f32_to_bf16_bits(X), gi.f32_to_bf16_bits(W), gi.f32_to_bf16_bits(R)
+    Yb, _, _ = oracle.run(Xb, np.zeros_like(Wb), None, None, dtype=oracle.BF16, act=oracle.ACT_NONE, scale_kind=oracle.SCALE_NONE,
+                          reduce=oracle.RED_MAXSUM, residual=Rb)
+    np.testing.assert_array_equal(Yb, gi.bf16_bits_to_f32(Rb).reshape(6, 14).astype(np.float64))
