@@ -32,7 +32,7 @@ _M1 = np.uint64(0xBF58476D1CE4E5B9)
 _M2 = np.uint64(0x94D049BB133111EB)
 _CHUNK = 1 << 20
 
-TENSOR_X, TENSOR_W, TENSOR_BIAS, TENSOR_SCALE = 1, 2, 3, 4
+TENSOR_X, TENSOR_W, TENSOR_BIAS, TENSOR_SCALE, TENSOR_RESIDUAL = 1, 2, 3, 4, 5
 
 # enum values of the operator descriptor (documented in include/fgr.h)
 DTYPE_F32, DTYPE_BF16 = 0, 1
@@ -136,6 +136,7 @@ class Problem:
     W: np.ndarray | None = None
     bias: np.ndarray | None = None
     scale_vec: np.ndarray | None = None
+    residual: np.ndarray | None = None    # [batch, M, N] in the dtype of X, added after activation and scale
     recipe: dict = field(default_factory=dict)
 
     @property
@@ -159,6 +160,8 @@ class Problem:
             b += self.bias.size * 4
         if self.scale_vec is not None:
             b += self.scale_vec.size * 4
+        if self.residual is not None:
+            b += self.batch * self.M * self.N * e
         if self.reduce == RED_SOFTMAX or self.write_y:
             b += self.batch * self.M * self.N * e
         b += self.batch * self.M * self.out_width * 4
@@ -171,7 +174,7 @@ def _store(a: np.ndarray, dtype: int) -> np.ndarray:
 
 def make_problem(name, batch, M, N, K, dtype, act, scale_kind, reduce, *, scale=1.0, write_y=0,
                  x_std=None, w_std=None, bias_range=(-0.1, 0.1), scale_range=(0.5, 1.5),
-                 bias_per_batch=0, seed=0, materialize=True, conv_taps=0, w_shared=0) -> Problem:
+                 bias_per_batch=0, seed=0, materialize=True, conv_taps=0, w_shared=0, residual_std=None) -> Problem:
     """Draws a problem with the value distributions of the named workloads.
 
     x_std / w_std default to 1/sqrt(K); bias ~ U(bias_range) (None -> no bias);
@@ -201,6 +204,8 @@ def make_problem(name, batch, M, N, K, dtype, act, scale_kind, reduce, *, scale=
         p.bias = uniform(seed, TENSOR_BIAS, nb, *bias_range)
     if scale_kind == SCALE_PER_COLUMN:
         p.scale_vec = uniform(seed, TENSOR_SCALE, N, *scale_range)
+    if residual_std is not None:
+        p.residual = _store(normal(seed, TENSOR_RESIDUAL, batch * M * N, residual_std), dtype).reshape(batch, M, N)
     return p
 
 

@@ -188,6 +188,19 @@ FGR_API int fgr_run_host(fgr_handle* h, const void* X, const void* W, const floa
                  void* Y, float* out);
 
 /*
+ * fgr_set_residual: a further epilogue of the operator class, the skip connection (fused chains of
+ * operators are what the paper's method rewrites, Section 1 and Section 4.1):
+ *     y = act(z + b) * s + R[batch, M, N]
+ * with R in the dtype of X / W / Y.  The residual is added after activation and scale, before the row
+ * reduction and before Y is rounded and stored.  R is a device pointer (16-byte aligned) used by every
+ * later fgr_run of this handle until it is set again; NULL removes it.  ldr / bsr: row and batch strides
+ * in elements, 0 = packed (N, M * ldr); multiples of 8 (bf16) / 4 (fp32).  R may be the same buffer as Y
+ * with the same strides (every element is read before it is written, by the same thread), except for
+ * SOFTMAX, whose second pass rewrites Y.  fgr_run_host and fgr_run_static take no residual.
+ */
+FGR_API int fgr_set_residual(fgr_handle* h, const void* R /*device*/, int64_t ldr, int64_t bsr);
+
+/*
  * fgr_get_status: synchronises the stream of the last fgr_run and returns the device status
  * word: FGR_OK, or FGR_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel gave up (the kernels
  * never trap and never spin without a limit), or FGR_ERR_CUDA if the stream reports an error.

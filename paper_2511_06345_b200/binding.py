@@ -24,7 +24,7 @@ FGR_PATH_UMMA_TF32X3 = 5
 
 FGR_STATIC_SCRATCH_BYTES = 4 << 20
 
-EXPORTS = ("fgr_plan", "fgr_create", "fgr_workspace_bytes", "fgr_get_plan", "fgr_run", "fgr_run_host", "fgr_run_static", "fgr_reduce_rows", "fgr_combine_shards",
+EXPORTS = ("fgr_plan", "fgr_create", "fgr_workspace_bytes", "fgr_get_plan", "fgr_run", "fgr_run_host", "fgr_run_static", "fgr_reduce_rows", "fgr_combine_shards", "fgr_set_residual",
            "fgr_get_status", "fgr_profile_enable", "fgr_profile_read", "fgr_destroy", "fgr_status_string", "fgr_path_name")
 
 
@@ -92,6 +92,7 @@ def lib() -> ctypes.CDLL:
         L.fgr_run_static.argtypes, L.fgr_run_static.restype = [ctypes.POINTER(fgr_desc)] + [vp] * 7, i
         L.fgr_reduce_rows.argtypes, L.fgr_reduce_rows.restype = [ctypes.POINTER(fgr_reduce_desc)] + [vp] * 4, i
         L.fgr_combine_shards.argtypes, L.fgr_combine_shards.restype = [ctypes.POINTER(fgr_shard_desc)] + [vp] * 4, i
+        L.fgr_set_residual.argtypes, L.fgr_set_residual.restype = [vp, vp, ctypes.c_int64, ctypes.c_int64], i
         L.fgr_get_status.argtypes, L.fgr_get_status.restype = [vp], i
         L.fgr_profile_enable.argtypes, L.fgr_profile_enable.restype = [vp, i], i
         L.fgr_profile_read.argtypes, L.fgr_profile_read.restype = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i)], i
@@ -199,6 +200,14 @@ def fgr_combine_shards(rows, shards, reduce, pairs, out, P_local=None, *, dtype=
     rc = lib().fgr_combine_shards(ctypes.byref(d), _addr(pairs), _addr(out), _addr(P_local), stream)
     if check and rc != FGR_OK:
         raise FgrError(rc, "fgr_combine_shards")
+    return rc
+
+
+def fgr_set_residual(h, R, ldr: int = 0, bsr: int = 0, check=True) -> int:
+    """Sets (or with ``R=None`` removes) the residual tensor added after activation and scale (a device pointer or tensor)."""
+    rc = lib().fgr_set_residual(h, _addr(R), int(ldr), int(bsr))
+    if check and rc != FGR_OK:
+        raise FgrError(rc, "fgr_set_residual")
     return rc
 
 

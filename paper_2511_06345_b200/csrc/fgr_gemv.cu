@@ -137,7 +137,8 @@ __global__ void __launch_bounds__(kGemvThreads, 1) gemv_kernel(const Params p, i
         float s = 1.0f;
         if (p.scale_kind == FGR_SCALE_PER_COLUMN) s = p.scale_vec[n];
         else if (p.scale_kind == FGR_SCALE_SCALAR) s = p.scale;
-        const float y = activation(p.act, z + (bias ? bias[n] : 0.0f)) * s;
+        float y = activation(p.act, z + (bias ? bias[n] : 0.0f)) * s;
+        if (p.R) y += __bfloat162float(static_cast<const __nv_bfloat16*>(p.R)[(long long)bt * p.bsr + (long long)lane * p.ldr + n]);
         if (p.write_y) Y[(long long)lane * p.ldy + n] = __float2bfloat16_rn(y);
         if (exp_kind) {
           const float mn = fmaxf(s0, y);

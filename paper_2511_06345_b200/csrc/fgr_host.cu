@@ -22,6 +22,9 @@ struct fgr_handle {
   CUtensorMap tmap_x, tmap_w;
   const void* cached_x;
   const void* cached_w;
+  // optional residual tensor (fgr_set_residual)
+  const void* residual;
+  long long ldr, bsr;
   // status plumbing
   void* last_workspace;
   cudaStream_t last_stream;
@@ -382,6 +385,7 @@ int fgr_run(fgr_handle* h, const void* X, const void* W, const float* bias, cons
 
   Params p = h->base;
   p.X = X; p.W = W; p.bias = bias; p.scale_vec = scale_vec; p.Y = Y; p.out = out;
+  p.R = h->residual; p.ldr = h->ldr; p.bsr = h->bsr;
   p.status = static_cast<int*>(workspace);
   p.parts = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes);
 
@@ -449,6 +453,19 @@ int fgr_run(fgr_handle* h, const void* X, const void* W, const float* bias, cons
   return rc;
 }
 
+int fgr_set_residual(fgr_handle* h, const void* R, int64_t ldr, int64_t bsr) {
+  if (!h || ldr < 0 || bsr < 0) return FGR_ERR_INVALID_ARG;
+  if (!R) { h->residual = nullptr; return FGR_OK; }
+  const fgr_desc& d = h->desc;
+  const int g = 16 / elem_bytes(d.dtype);
+  const long long l = ldr ? ldr : d.N, b = bsr ? bsr : (long long)d.M * l;
+  if (l < d.N || (d.batch > 1 && b < (long long)(d.M - 1) * l + d.N)) return FGR_ERR_INVALID_ARG;
+  if (l % g || b % g) return FGR_ERR_UNSUPPORTED;
+  if (!aligned16(R)) return FGR_ERR_INVALID_ARG;
+  h->residual = R; h->ldr = l; h->bsr = b;
+  return FGR_OK;
+}
+
 int fgr_get_status(fgr_handle* h) {
   if (!h) return FGR_ERR_INVALID_ARG;
   if (!h->ran) return FGR_OK;
@@ -478,6 +495,7 @@ int fgr_run_host(fgr_handle* h, const void* X, const void* W, const float* bias,
   const bool need_y = d.write_y || softmax;
   if ((need_y && !Y) || (!softmax && !out)) return FGR_ERR_INVALID_ARG;
   if (d.scale_kind == FGR_SCALE_PER_COLUMN && !scale_vec) return FGR_ERR_INVALID_ARG;
+  if (h->residual) return FGR_ERR_UNSUPPORTED;   // the residual is a device tensor: use fgr_run
   const size_t e = (size_t)elem_bytes(d.dtype);
   // extents in bytes of each buffer as laid out by the descriptor's strides
   const size_t want[7] = {

@@ -27,6 +27,8 @@ struct Params {
   const float* bias;
   const float* scale_vec;
   void* Y;
+  const void* R;       // residual tensor [batch, M, N] in the dtype of Y, added after activation and scale; may be null
+  long long ldr, bsr;  // its row and batch strides in elements
   float* out;
   float* parts;        // [batch * M][parts_per_row][2] split-N partial pairs
   int* status;         // device status word (0 = ok)

@@ -25,6 +25,8 @@ __device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
   f.w = __uint_as_float(r.y & 0xffff0000u);
   return f;
 }
+__device__ __forceinline__ float to_float(float v) { return v; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
 __device__ __forceinline__ void store4(float* p, float a, float b, float c, float d) {
   *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d);
 }
@@ -128,6 +130,7 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(const Params p) {
     }
   }
   T* Y = static_cast<T*>(p.Y) + (long long)bt * p.bsy;
+  const T* Rres = p.R ? static_cast<const T*>(p.R) + (long long)bt * p.bsr : nullptr;
   const bool meanvar = p.reduce == FGR_RED_MEANVAR;
   const bool exp_kind = p.reduce != FGR_RED_MAXSUM && !meanvar;
   const bool store_y = p.write_y && p.reduce != FGR_RED_SOFTMAX;
@@ -141,6 +144,7 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(const Params p) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       y[j] = activation(p.act, acc[i][j] + bj[j]) * sj[j];
+      if (Rres && cols_ok && m < p.M) y[j] += to_float(Rres[(long long)m * p.ldr + nc + j]);
       if (cols_ok) { mx = fmaxf(mx, y[j]); sm += y[j]; }
     }
     if (store_y && cols_ok && m < p.M) store4(Y + (long long)m * p.ldy + nc, y[0], y[1], y[2], y[3]);

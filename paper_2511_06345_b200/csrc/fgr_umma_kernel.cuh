@@ -272,6 +272,31 @@ __device__ __forceinline__ void store_f32x16(float* dst, const float* y, int nv)
     if (4 * q < nv) *reinterpret_cast<float4*>(dst + 4 * q) = make_float4(y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]);
 }
 
+// y[0..16) += f * R[0..16): the residual tensor's elements for 16 columns of one row, of which the first nv
+// (bf16: 8 or 16; fp32: a multiple of 4) are inside the matrix.
+__device__ __forceinline__ void add_residual16(float* y, const __nv_bfloat16* r, int nv, float f) {
+#pragma unroll
+  for (int h = 0; h < 2; ++h)
+    if (h == 0 || nv >= kChunk) {
+      const uint4 v = *reinterpret_cast<const uint4*>(r + 8 * h);
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        y[8 * h + 2 * i] = fmaf(f, __uint_as_float(w[i] << 16), y[8 * h + 2 * i]);
+        y[8 * h + 2 * i + 1] = fmaf(f, __uint_as_float(w[i] & 0xffff0000u), y[8 * h + 2 * i + 1]);
+      }
+    }
+}
+__device__ __forceinline__ void add_residual16(float* y, const float* r, int nv, float f) {
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    if (4 * q < nv) {
+      const float4 v = *reinterpret_cast<const float4*>(r + 4 * q);
+      y[4 * q] = fmaf(f, v.x, y[4 * q]); y[4 * q + 1] = fmaf(f, v.y, y[4 * q + 1]);
+      y[4 * q + 2] = fmaf(f, v.z, y[4 * q + 2]); y[4 * q + 3] = fmaf(f, v.w, y[4 * q + 3]);
+    }
+}
+
 // Work unit t -> (batch, first row of this CTA, first column).  A unit is one 128-row tile, or for
 // a CTA pair a 256-row tile of which CTA `rank` owns rows [128 rank, 128 rank + 128).
 struct TileCoord { int bt, m0, n0; };
@@ -586,6 +611,10 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * 256u;
       using OutT = typename std::conditional<TF32, float, __nv_bfloat16>::type;
       OutT* yrow = static_cast<OutT*>(p.Y) + (long long)c.bt * p.bsy + (long long)m * p.ldy + c.n0;
+      // the residual row (added after activation and scale; in log2 units where the epilogue works in them)
+      const OutT* rrow = p.R ? static_cast<const OutT*>(p.R) + (long long)c.bt * p.bsr + (long long)m * p.ldr + c.n0 : nullptr;
+      const bool use_r = rrow != nullptr && row_ok;
+      constexpr float kResF = V::kFoldLog2e ? kLog2e : 1.0f;
       // is column j of a 16-column chunk with nv real columns inside the matrix?  (bf16: N is a multiple
       // of 8, so a ragged chunk has exactly 8; fp32: a multiple of 4)
       auto real = [](int j, int nv) { return TF32 ? j < nv : (j < 8 || nv >= kChunk); };
@@ -614,6 +643,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
                 for (int j = 0; j < kChunk; ++j) S[kChunk * q + j] += __uint_as_float(ra[j]);
               }
               apply16f<ACT, SC>(S + kChunk * q, bias_s + kChunk * q, scale_s + kChunk * q, y);
+              if (use_r) add_residual16(y, rrow + cc, c_lim - cc, kResF);
               f(y, cc, c_lim - cc);
             }
           }
@@ -625,9 +655,11 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
           if (second) tcgen05_ld16_issue(taddr + cc + kChunk, rb);
           tcgen05_wait_ld();
           apply16<ACT, SC>(ra, bias_s + (cc - c_begin), scale_s + (cc - c_begin), y);
+          if (use_r) add_residual16(y, rrow + cc, c_lim - cc, kResF);
           f(y, cc, c_lim - cc);
           if (second) {
             apply16<ACT, SC>(rb, bias_s + (cc + kChunk - c_begin), scale_s + (cc + kChunk - c_begin), y);
+            if (use_r) add_residual16(y, rrow + cc + kChunk, c_lim - cc - kChunk, kResF);
             f(y, cc + kChunk, c_lim - cc - kChunk);
           }
         }

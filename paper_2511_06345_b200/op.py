@@ -40,8 +40,10 @@ class FusedGemmReduce:
     def path(self) -> str:
         return B.fgr_path_name(self.plan.path)
 
-    def __call__(self, X, W, bias=None, scale_vec=None, Y=None, out=None):
+    def __call__(self, X, W, bias=None, scale_vec=None, Y=None, out=None, residual=None):
         d = self.desc
+        B.fgr_set_residual(self.handle, residual)     # [batch, M, N] in the operator's dtype, packed; None = none
+        self._residual = residual                     # keeps the tensor alive while the handle points at it
         if Y is None and self.need_y:
             Y = torch.empty((d.batch, d.M, d.N), dtype=self.tdtype, device=self.device)
         if out is None and self.out_shape is not None:

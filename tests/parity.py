@@ -46,8 +46,12 @@ def run_gpu(p: gi.Problem, force_path=0, force_tile_n=0, device=0, tensors=None,
                              force_path=force_path, force_tile_n=force_tile_n, force_cta_pair=force_cta_pair, force_ksub=force_ksub,
                              conv_taps=p.conv_taps, w_shared=p.w_shared)
     X, W, b, s = tensors if tensors is not None else to_device(p, "cuda:%d" % device)
+    R = None
+    if getattr(p, "residual", None) is not None:
+        t = torch.from_numpy(np.ascontiguousarray(p.residual))
+        R = (t.view(torch.int16).view(torch.bfloat16) if p.dtype == gi.DTYPE_BF16 else t).to("cuda:%d" % device)
     for _ in range(repeat):
-        Y, out = op(X, W, b, s)
+        Y, out = op(X, W, b, s, residual=R)
     st = op.status()
     assert st == fgr.FGR_OK, fgr.fgr_status_string(st)
     plan = op.plan.as_dict()
