@@ -18,9 +18,9 @@ cudaError_t launch_umma(const Params& p, const void* tmap_x, const void* tmap_w,
                         cudaStream_t stream) {
   const bool softmax = p.reduce == FGR_RED_SOFTMAX;
   const bool exp_kind = p.reduce == FGR_RED_LSE || p.reduce == FGR_RED_SOFTMAX || p.reduce == FGR_RED_MAX_SUMEXP;
-  const bool wy = p.write_y && !softmax;
+  const bool wy = softmax ? p.R != nullptr : p.write_y != 0;   // softmax: the variant compiled with the residual add
   // exp kinds that do not store y fold log2(e) into the staged scale vector, so they always multiply
-  const bool sc = (exp_kind && !wy) || p.scale_kind != FGR_SCALE_NONE;
+  const bool sc = (exp_kind && (softmax || !wy)) || p.scale_kind != FGR_SCALE_NONE;
   switch (p.act) {
     case FGR_ACT_NONE: return umma_launch_act_none(sc, p.reduce, wy, p, tmap_x, tmap_w, grid, smem_bytes, stream);
     case FGR_ACT_RELU: return umma_launch_act_relu(sc, p.reduce, wy, p, tmap_x, tmap_w, grid, smem_bytes, stream);

@@ -312,11 +312,14 @@ __device__ __forceinline__ TileCoord tile_coord(long long t, const Params& p, in
 
 // Compile-time description of one epilogue variant.
 //   ACT : fgr_act          SC : multiply by the staged scale vector
-//   RED : fgr_reduce       WY : store y as bf16 (ignored for softmax, which always stores)
+//   RED : fgr_reduce       WY : store y as bf16 (softmax always stores; there WY selects the variant with a residual)
 template <int ACT, bool SC, int RED, bool WY>
 struct Variant {
   static constexpr bool kExp = RED == FGR_RED_LSE || RED == FGR_RED_SOFTMAX || RED == FGR_RED_MAX_SUMEXP;
   static constexpr bool kMeanVar = RED == FGR_RED_MEANVAR;
+  // the residual add is compiled into every variant but plain softmax, whose WY = true twin carries it
+  // (its two passes over the accumulator are the most register-hungry epilogue)
+  static constexpr bool kResidual = RED != FGR_RED_SOFTMAX || WY;
   static constexpr bool kSoftmax = RED == FGR_RED_SOFTMAX;
   static constexpr bool kStoreY = WY && !kSoftmax;
   // exp kinds work in log2 units; when y itself is not stored the factor log2(e) is folded into
@@ -613,7 +616,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
       OutT* yrow = static_cast<OutT*>(p.Y) + (long long)c.bt * p.bsy + (long long)m * p.ldy + c.n0;
       // the residual row (added after activation and scale; in log2 units where the epilogue works in them)
       const OutT* rrow = p.R ? static_cast<const OutT*>(p.R) + (long long)c.bt * p.bsr + (long long)m * p.ldr + c.n0 : nullptr;
-      const bool use_r = rrow != nullptr && row_ok;
+      const bool use_r = V::kResidual && rrow != nullptr && row_ok;
       constexpr float kResF = V::kFoldLog2e ? kLog2e : 1.0f;
       // is column j of a 16-column chunk with nv real columns inside the matrix?  (bf16: N is a multiple
       // of 8, so a ragged chunk has exactly 8; fp32: a multiple of 4)
@@ -793,7 +796,7 @@ cudaError_t prepare_one() {
   X(false, FGR_RED_MAXSUM, false) X(false, FGR_RED_MAXSUM, true) X(true, FGR_RED_MAXSUM, false)   \
   X(true, FGR_RED_MAXSUM, true) X(true, FGR_RED_LSE, false) X(false, FGR_RED_LSE, true)           \
   X(true, FGR_RED_LSE, true) X(true, FGR_RED_MAX_SUMEXP, false) X(false, FGR_RED_MAX_SUMEXP, true) \
-  X(true, FGR_RED_MAX_SUMEXP, true) X(true, FGR_RED_SOFTMAX, false)                               \
+  X(true, FGR_RED_MAX_SUMEXP, true) X(true, FGR_RED_SOFTMAX, false) X(true, FGR_RED_SOFTMAX, true) \
   X(false, FGR_RED_MEANVAR, false) X(false, FGR_RED_MEANVAR, true) X(true, FGR_RED_MEANVAR, false) \
   X(true, FGR_RED_MEANVAR, true)
 
