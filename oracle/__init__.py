@@ -145,31 +145,31 @@ def run(X, W, bias, scale_vec, *, dtype, act, scale_kind, reduce, scale=1.0, bia
     return Y, out, rc
 
 
-def conv1d_windows(x, taps: int):
+def conv1d_windows(x, taps: int, stride: int = 1):
     """Rows of the 1-D convolution written out as a matrix (no arithmetic, only copies).
 
     The operator category "convolution" (Section 1; Section 4.1, Datasets; the 1-D case is the paper's
     case study, Section 4.4): for a channels-last input x [batch, L, C] and a filter bank
-    w [N, taps, C] (stride 1, no padding, no dilation),
+    w [N, taps, C] (no padding, no dilation, stride s),
 
-        z[b, l, n] = sum_{r = 0 .. taps-1} sum_{c = 0 .. C-1} x[b, l + r, c] * w[n, r, c],   l = 0 .. L - taps,
+        z[b, l, n] = sum_{r = 0 .. taps-1} sum_{c = 0 .. C-1} x[b, l s + r, c] * w[n, r, c],   l = 0 .. (L - taps) // s,
 
-    which is the product of the window matrix  A[b, l, r * C + c] = x[b, l + r, c]  with  w  viewed as
-    [N, taps * C].  This returns A [batch, L - taps + 1, taps * C]; ``run`` on (A, w) is then the
+    which is the product of the window matrix  A[b, l, r * C + c] = x[b, l s + r, c]  with  w  viewed as
+    [N, taps * C].  This returns A [batch, (L - taps) // s + 1, taps * C]; ``run`` on (A, w) is then the
     definition of the fused convolution + epilogue + reduction over the output channels.
     """
     x = np.ascontiguousarray(x)
     if x.ndim == 2:
         x = x[None]
     batch, L, C = x.shape
-    if taps < 1 or taps > L:
-        raise ValueError("taps must be in 1..L")
-    Lo = L - taps + 1
+    if taps < 1 or taps > L or stride < 1:
+        raise ValueError("taps must be in 1..L and stride >= 1")
+    Lo = (L - taps) // stride + 1
     A = np.empty((batch, Lo, taps * C), dtype=x.dtype)
     for b in range(batch):
         for l in range(Lo):
             for r in range(taps):
-                A[b, l, r * C:(r + 1) * C] = x[b, l + r, :]
+                A[b, l, r * C:(r + 1) * C] = x[b, l * stride + r, :]
     return A
 
 
@@ -178,7 +178,7 @@ def run_problem(p, rows=None, want_y=True, nthreads=0):
     With ``p.conv_taps > 1``, ``p.X`` is the channels-last input [batch, L, C] of a 1-D convolution and
     ``p.W`` its filters [batch, N, taps * C]."""
     if getattr(p, "conv_taps", 0) > 1:
-        return run(conv1d_windows(p.X, p.conv_taps), p.W, p.bias, p.scale_vec, dtype=p.dtype, act=p.act,
+        return run(conv1d_windows(p.X, p.conv_taps, getattr(p, "conv_stride", 1) or 1), p.W, p.bias, p.scale_vec, dtype=p.dtype, act=p.act,
                    scale_kind=p.scale_kind, reduce=p.reduce, scale=p.scale, bias_per_batch=p.bias_per_batch,
                    rows=rows, want_y=want_y, nthreads=nthreads, residual=getattr(p, "residual", None))
     return run(p.X, p.W, p.bias, p.scale_vec, dtype=p.dtype, act=p.act, scale_kind=p.scale_kind,

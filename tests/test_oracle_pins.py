@@ -519,3 +519,17 @@ def test_residual_closed_forms_and_library():
     Yb, _, _ = oracle.run(Xb, np.zeros_like(Wb), None, None, dtype=oracle.BF16, act=oracle.ACT_NONE, scale_kind=oracle.SCALE_NONE,
                           reduce=oracle.RED_MAXSUM, residual=Rb)
     np.testing.assert_array_equal(Yb, gi.bf16_bits_to_f32(Rb).reshape(6, 14).astype(np.float64))
+
+
+def test_conv1d_stride_matches_library_fp64():
+    B, L, C, N, R, S = 2, 23, 4, 3, 3, 2
+    x = _rand((B, L, C), 54)
+    w = _rand((N, R, C), 55, tid=8)
+    A = oracle.conv1d_windows(x, R, stride=S)
+    assert A.shape == (B, (L - R) // S + 1, R * C)
+    np.testing.assert_array_equal(A[1, 4], x[1, 8:11].reshape(-1))            # window l = 4 starts at sample l * S = 8
+    Y, _, _ = oracle.run(A, np.broadcast_to(w.reshape(1, N, R * C), (B, N, R * C)).copy(), None, None, dtype=oracle.F32,
+                         act=oracle.ACT_NONE, scale_kind=oracle.SCALE_NONE, reduce=oracle.RED_MAXSUM)
+    ref = torch.nn.functional.conv1d(torch.from_numpy(x).double().permute(0, 2, 1), torch.from_numpy(w).double().permute(0, 2, 1),
+                                     stride=S).permute(0, 2, 1).reshape(-1, N)
+    np.testing.assert_allclose(Y, ref.numpy(), rtol=1e-13, atol=1e-15)
