@@ -131,7 +131,8 @@ class Problem:
     write_y: int = 0
     bias_per_batch: int = 0
     w_shared: int = 0      # 1: W is [1, N, K], one matrix for every batch element
-    conv_taps: int = 0     # R > 1: 1-D convolution; X is then [batch, M + R - 1, K / R] (channels last)
+    conv_taps: int = 0     # R > 1: 1-D convolution; X is then [batch, (M - 1) * stride + R, K / R] (channels last)
+    conv_stride: int = 1
     X: np.ndarray | None = None
     W: np.ndarray | None = None
     bias: np.ndarray | None = None
@@ -155,7 +156,8 @@ class Problem:
         """Algorithmic minimum traffic: every operand read once, every output written once."""
         e = self.elem_bytes
         taps = max(self.conv_taps, 1)
-        b = (self.batch * (self.M + taps - 1) * (self.K // taps) + (1 if self.w_shared else self.batch) * self.N * self.K) * e
+        x_elems = (self.M - 1) * min(self.conv_stride * (self.K // taps), self.K) + self.K if taps > 1 else self.M * self.K
+        b = (self.batch * x_elems + (1 if self.w_shared else self.batch) * self.N * self.K) * e
         if self.bias is not None:
             b += self.bias.size * 4
         if self.scale_vec is not None:
@@ -174,7 +176,7 @@ def _store(a: np.ndarray, dtype: int) -> np.ndarray:
 
 def make_problem(name, batch, M, N, K, dtype, act, scale_kind, reduce, *, scale=1.0, write_y=0,
                  x_std=None, w_std=None, bias_range=(-0.1, 0.1), scale_range=(0.5, 1.5),
-                 bias_per_batch=0, seed=0, materialize=True, conv_taps=0, w_shared=0, residual_std=None) -> Problem:
+                 bias_per_batch=0, seed=0, materialize=True, conv_taps=0, w_shared=0, residual_std=None, conv_stride=1) -> Problem:
     """Draws a problem with the value distributions of the named workloads.
 
     x_std / w_std default to 1/sqrt(K); bias ~ U(bias_range) (None -> no bias);
@@ -183,7 +185,7 @@ def make_problem(name, batch, M, N, K, dtype, act, scale_kind, reduce, *, scale=
     x_std = 1.0 / math.sqrt(K) if x_std is None else x_std
     w_std = 1.0 / math.sqrt(K) if w_std is None else w_std
     p = Problem(name, batch, M, N, K, dtype, act, scale_kind, reduce, scale=float(scale),
-                write_y=write_y, bias_per_batch=bias_per_batch, conv_taps=conv_taps, w_shared=w_shared,
+                write_y=write_y, bias_per_batch=bias_per_batch, conv_taps=conv_taps, w_shared=w_shared, conv_stride=conv_stride,
                 recipe=dict(seed=seed, x_std=x_std, w_std=w_std, bias_range=bias_range,
                             scale_range=scale_range if scale_kind == SCALE_PER_COLUMN else None))
     if not materialize:
@@ -193,7 +195,7 @@ def make_problem(name, batch, M, N, K, dtype, act, scale_kind, reduce, *, scale=
             p.scale_vec = np.empty(N, dtype=np.float32)
         return p
     if conv_taps > 1:      # the input signal itself; the operator reads overlapping windows of it
-        L, C = M + conv_taps - 1, K // conv_taps
+        L, C = (M - 1) * conv_stride + conv_taps, K // conv_taps
         p.X = _store(normal(seed, TENSOR_X, batch * L * C, x_std), dtype).reshape(batch, L, C)
     else:
         p.X = _store(normal(seed, TENSOR_X, batch * M * K, x_std), dtype).reshape(batch, M, K)

@@ -107,8 +107,10 @@ typedef struct fgr_desc {
                               W the filters [batch, N, R * C] (tap-major, channel-minor), stride 1, no padding:
                                 z[b, l, n] = sum_r sum_c X[b, l + r, c] * W[n, r * C + c],   l = 0 .. M - 1.
                               Output row l of the GEMM reads the K = R * C contiguous elements that start at
-                              X[b, l, 0], so the rows of the implicit matrix overlap: ldx is C (0 or C; channel
-                              padding is not supported) and bsx defaults to L * C; nothing is copied or unfolded.  K % R == 0 and C a multiple of 8 (bf16)
+                              X[b, l, 0], so the rows of the implicit matrix overlap: ldx = 0 means C (stride 1); a
+                              convolution of stride s has ldx = s * C (then L = (M - 1) * s + R; any multiple of C is
+                              taken as such a stride, channel padding is not supported); bsx defaults to the signal
+                              length times C; nothing is copied or unfolded.  K % R == 0 and C a multiple of 8 (bf16)
                               / 4 (fp32).  fgr_run_static takes plain GEMMs only. */
   int32_t w_shared;        /* 0: W is [batch, N, K] (one weight matrix per batch element).  1: W is one [N, K] matrix
                               used by every batch element (bsw is ignored) - a filter bank shared by all signals of

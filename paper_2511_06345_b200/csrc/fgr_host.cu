@@ -63,7 +63,8 @@ Resolved resolve_strides(const fgr_desc& d) {
   r.ldx = d.ldx ? d.ldx : d.K / taps;
   r.ldw = d.ldw ? d.ldw : d.K;
   r.ldy = d.ldy ? d.ldy : d.N;
-  r.bsx = d.bsx ? d.bsx : (long long)(d.M + taps - 1) * r.ldx;
+  // (a strided convolution has ldx = stride * C: its signal is (M - 1) * stride + taps samples of C channels)
+  r.bsx = d.bsx ? d.bsx : (taps > 1 ? (long long)(d.M - 1) * r.ldx + d.K : (long long)d.M * r.ldx);
   r.bsw = d.w_shared ? 0 : (d.bsw ? d.bsw : (long long)d.N * r.ldw);   // shared W: every batch reads the same matrix
   r.bsy = d.bsy ? d.bsy : (long long)d.M * r.ldy;
   return r;
@@ -91,7 +92,8 @@ int validate(const fgr_desc* d) {
   if ((d->K / taps) % g) return FGR_ERR_UNSUPPORTED;
   const Resolved r = resolve_strides(*d);
   if (r.ldx < d->K / taps || r.ldw < d->K || r.ldy < d->N) return FGR_ERR_INVALID_ARG;
-  if (taps > 1 && r.ldx != d->K / taps) return FGR_ERR_UNSUPPORTED;   // a window must be K contiguous elements
+  // a window must be K contiguous elements: the row stride is the convolution's stride times C, never a padded C
+  if (taps > 1 && r.ldx % (d->K / taps) != 0) return FGR_ERR_UNSUPPORTED;
   if (r.ldx % g || r.ldw % g || r.ldy % g || r.bsx % g || r.bsw % g || r.bsy % g) return FGR_ERR_UNSUPPORTED;
   if (d->batch > 1 && (r.bsx < (long long)(d->M - 1) * r.ldx + d->K || (!d->w_shared && r.bsw < (long long)(d->N - 1) * r.ldw + d->K) ||
                        r.bsy < (long long)(d->M - 1) * r.ldy + d->N))
@@ -106,7 +108,9 @@ int validate(const fgr_desc* d) {
 double min_bytes(const fgr_desc& d) {
   const double e = elem_bytes(d.dtype);
   const int taps = d.conv_taps > 1 ? d.conv_taps : 1;   // a convolution's input is read once, not once per tap
-  double b = ((double)d.batch * (d.M + taps - 1) * (d.K / taps) + (double)(d.w_shared ? 1 : d.batch) * d.N * d.K) * e;
+  const Resolved rs = resolve_strides(d);
+  const double x_elems = taps > 1 ? (double)(d.M - 1) * (rs.ldx < d.K ? rs.ldx : d.K) + d.K : (double)d.M * d.K;   // samples actually read
+  double b = ((double)d.batch * x_elems + (double)(d.w_shared ? 1 : d.batch) * d.N * d.K) * e;
   b += 4.0 * d.N * (d.bias_per_batch ? d.batch : 1);   // bias (counted whether or not one is passed)
   if (d.scale_kind == FGR_SCALE_PER_COLUMN) b += 4.0 * d.N;
   if (d.write_y || d.reduce == FGR_RED_SOFTMAX) b += (double)d.batch * d.M * d.N * e;

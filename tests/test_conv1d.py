@@ -107,3 +107,28 @@ def test_conv1d_host_buffers(cuda_device):
     fgr.fgr_destroy(h)
     Yf = gi.bf16_bits_to_f32(Y.numpy().view(np.uint16)).astype(np.float64).reshape(p.batch * p.M, p.N)
     compare(p, Yf, out.numpy().astype(np.float64))
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("case", [(gi.DTYPE_BF16, fgr.FGR_PATH_UMMA_TILED, 2), (gi.DTYPE_BF16, fgr.FGR_PATH_UMMA_STREAM_W, 3),
+                                  (gi.DTYPE_BF16, fgr.FGR_PATH_SIMT, 2), (gi.DTYPE_F32, fgr.FGR_PATH_UMMA_TF32X3, 2),
+                                  (gi.DTYPE_BF16, fgr.FGR_PATH_UMMA_TILED, 5)])
+def test_conv1d_strided(cuda_device, case):
+    """Stride s: the row stride of the implicit matrix is s * C (for s > R samples are skipped altogether)."""
+    from parity import compare, run_gpu
+    dtype, path, stride = case
+    B, M, N, C, R = 2, 130, 264, 24, 3
+    p = gi.make_problem("conv", B, M, N, R * C, dtype, gi.ACT_GELU_TANH, gi.SCALE_NONE, gi.RED_LSE, write_y=1, x_std=1.0,
+                        w_std=2.0 / np.sqrt(R * C), seed=21, conv_taps=R, conv_stride=stride, w_shared=1)
+    assert p.X.shape == (B, (M - 1) * stride + R, C)
+    Y, out, plan = run_gpu(p, force_path=path)
+    assert plan["path"] == path
+    kw = {}
+    if path == fgr.FGR_PATH_UMMA_TF32X3:
+        from test_tf32x3 import _slack
+        import copy, oracle
+        q = copy.copy(p)
+        q.X, q.conv_taps, q.W = oracle.conv1d_windows(p.X, R, stride), 0, np.broadcast_to(p.W, (B,) + p.W.shape[1:])
+        ys, os_, yr = _slack(q)
+        kw = dict(y_slack=ys, out_slack=os_, y_rel_slack=yr)
+    compare(p, Y, out, tcgen05=dtype == gi.DTYPE_BF16 and path != fgr.FGR_PATH_SIMT, **kw)
