@@ -144,3 +144,24 @@ def test_null_and_misaligned_pointers_are_rejected(cuda_device):
     assert run(X, W, b, s, Y, out, ws.data_ptr() + 64, n) == fgr.FGR_ERR_WORKSPACE
     assert run(X, W, b, s, Y, out, ws, n) == fgr.FGR_OK and fgr.fgr_get_status(h) == fgr.FGR_OK
     fgr.fgr_destroy(h)
+
+
+@pytest.mark.parametrize("path", [fgr.FGR_PATH_UMMA_TILED, fgr.FGR_PATH_UMMA_STREAM_W, fgr.FGR_PATH_SIMT])
+@pytest.mark.parametrize("red", [gi.RED_LSE, gi.RED_SOFTMAX, gi.RED_MAXSUM])
+def test_non_finite_inputs_stay_in_their_rows(cuda_device, path, red):
+    """NaN and infinities in X are outside the contract, but they must neither stall a kernel nor leak
+    into other rows: the run completes with a clean device status, the affected rows come out
+    non-finite, every other row still matches the oracle."""
+    p = _base(128, 520, 136, red, act=gi.ACT_GELU_TANH, seed=91)
+    X = gi.bf16_bits_to_f32(p.X).reshape(p.X.shape).copy()
+    X[0, 3, 17] = np.nan
+    X[0, 70, 5] = np.inf
+    X[0, 71, :] = -np.inf
+    p.X = gi.f32_to_bf16_bits(X).reshape(X.shape)
+    Y, out, plan = run_gpu(p, force_path=path)           # run_gpu asserts the device status word
+    bad = [3, 70, 71]
+    good = np.array([r for r in range(p.M) if r not in bad])
+    compare(p, Y, out, rows=good, tcgen05=path != fgr.FGR_PATH_SIMT)
+    assert not np.isfinite(Y[3]).all()
+    if out is not None:
+        assert not np.isfinite(out[3]).all()
