@@ -12,10 +12,17 @@
  *     FGR_RED_SOFTMAX    P[m, n]   = exp(y[m, n]) / sum_n exp(y[m, n])      (written in Y's slot)
  *     FGR_RED_MAXSUM     out[m, :] = ( max_n y , sum_n y )
  *     FGR_RED_MAX_SUMEXP out[m, :] = ( max_n y , sum_n exp(y - max_n y) )
+ *     FGR_RED_MEANVAR    out[m, :] = ( mean_n y , (1/N) sum_n (y - mean)^2 )
+ *
+ * Variations of the same operator (each documented where it is declared): a residual tensor added to
+ * y (fgr_set_residual), one weight matrix shared by all batch elements (fgr_desc.w_shared), 1-D
+ * convolution as an implicit GEMM (fgr_desc.conv_taps), fp32 problems on tensor cores
+ * (FGR_PATH_UMMA_TF32X3), N sharded over several GPUs (fgr_combine_shards), and the reductions alone on
+ * a given matrix (fgr_reduce_rows).
  *
  * Where this comes from.  The paper's task statement is: given the reference operator's inputs,
  * produce the same outputs, faster (Section 3.1, Verifier; Section 3.3), for operators of the
- * categories "matrix multiplication, element-wise and reduction" (Section 1; Section 4.1,
+ * categories "matrix multiplication, convolution, element-wise and reduction" (Section 1; Section 4.1,
  * Datasets).  The paper prints no formula for any operator; the formulas above are the plain
  * definitions of a linear layer, the activation, a scale and a last-dimension reduction.
  *
