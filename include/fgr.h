@@ -182,6 +182,8 @@ FGR_API int fgr_get_plan(const fgr_handle* h, fgr_plan_info* info /*host, out*/)
  *              must not share a workspace.
  *   cuda_stream  a cudaStream_t passed as void*; NULL = the default stream
  * Results are bit-identical from run to run (the merge order is fixed; no floating atomics).
+ * The call only enqueues kernels; after one ordinary call with the same pointers (which clears the
+ * workspace's status word and encodes the tensor maps) it can be captured into a CUDA graph.
  */
 FGR_API int fgr_run(fgr_handle* h, const void* X, const void* W, const float* bias, const float* scale_vec,
             void* Y, float* out, void* workspace, size_t workspace_bytes, void* cuda_stream);

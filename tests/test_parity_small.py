@@ -277,3 +277,30 @@ def test_shared_weights_plain_gemm(cuda_device):
     Y, out, plan = run_gpu(p)
     assert plan["path"] == fgr.FGR_PATH_SIMT_GEMV
     compare(p, Y, out)
+
+
+def test_run_inside_a_cuda_graph(cuda_device):
+    """fgr_run only enqueues kernels (with programmatic dependent launch between them), so after one
+    ordinary call (which clears the workspace's status word and encodes the tensor maps) it can be
+    captured into a CUDA graph; replays give bit-identical results."""
+    p = gi.make_problem("t", 2, 300, 520, 200, gi.DTYPE_BF16, gi.ACT_GELU_TANH, gi.SCALE_NONE, gi.RED_LSE, write_y=1, seed=77)
+    X, W, b, s = to_device(p)
+    op = fgr.FusedGemmReduce(p.batch, p.M, p.N, p.K, p.dtype, p.act, p.scale_kind, p.reduce, write_y=1, device=0)
+    Y = torch.empty((p.batch, p.M, p.N), dtype=torch.bfloat16, device="cuda")
+    out = torch.empty((p.batch * p.M,), dtype=torch.float32, device="cuda")
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        op(X, W, b, s, Y=Y, out=out)
+        stream.synchronize()
+        Y0, out0 = Y.clone(), out.clone()
+        Y.zero_(); out.zero_()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for _ in range(3):
+                op(X, W, b, s, Y=Y, out=out)
+        g.replay()
+        stream.synchronize()
+    assert op.status() == fgr.FGR_OK
+    assert torch.equal(Y, Y0) and torch.equal(out, out0)
+    compare(p, Y.float().cpu().numpy().astype(np.float64).reshape(p.batch * p.M, p.N), out.cpu().numpy().astype(np.float64).reshape(-1, 1))
+    op.close()
