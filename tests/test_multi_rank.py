@@ -74,3 +74,20 @@ def test_reference_arm_prints_the_contract_line():
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["value"] == line["value"]
     assert line["config"]["workload"] == "c1" and line["vs_baseline"] is None
+
+
+def test_bench_extra_workloads_are_well_formed():
+    """The extra bench legs resolve to problems of the documented shapes (no data is generated here)."""
+    sys.path.insert(0, ROOT)
+    import bench
+    import fgr_inputs as gi
+    f2 = bench.make_cfg("f2", materialize=False)
+    assert (f2.dtype, f2.M, f2.N, f2.K, f2.write_y) == (gi.DTYPE_F32, 4096, 4096, 4096, 1)
+    v2 = bench.make_cfg("v2", materialize=False)
+    assert (v2.batch, v2.M, v2.N, v2.K, v2.conv_taps, v2.w_shared) == (8, 2048, 4096, 2048, 4, 1)
+    assert v2.flop == 2.0 * 8 * 2048 * 4096 * 2048
+    g2 = bench.make_cfg("g2", materialize=False)
+    assert (g2.M, g2.N, g2.K) == (2, 16384, 8192)
+    for name in ("c2", "c3", "c4", "c5", "f2", "v2", "g2"):
+        assert name in bench.TRAFFIC
+    assert set(bench.NSHARD_CONFIGS) == {"c4n"} and "r_max_long" in bench.REDUCE_CONFIGS
