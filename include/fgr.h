@@ -74,7 +74,7 @@ typedef enum { FGR_SCALE_NONE = 0, FGR_SCALE_SCALAR = 1, FGR_SCALE_PER_COLUMN = 
 typedef enum { FGR_RED_LSE = 0, FGR_RED_SOFTMAX = 1, FGR_RED_MAXSUM = 2, FGR_RED_MAX_SUMEXP = 3,
                /* (mean, population variance) of y over N: the row statistics of a normalisation layer.  Computed
                   per tile in two passes and merged pairwise (mean, sum of squared deviations), never as
-                  E[y^2] - E[y]^2.  Not on the FGR_PATH_SIMT_GEMV path and not in fgr_combine_shards. */
+                  E[y^2] - E[y]^2.  Not on the FGR_PATH_SIMT_GEMV path. */
                FGR_RED_MEANVAR = 6 } fgr_reduce;
 
 /* Execution paths (fgr_plan_info.path, fgr_desc.force_path). */
@@ -283,8 +283,11 @@ FGR_API int fgr_reduce_rows(const fgr_reduce_desc* desc /*host*/, const void* A,
  * problem statement is unchanged: the same outputs as the unsharded operator (Section 3.1,
  * Verifier; Section 3.3).  Protocol, per GPU g of G:
  *   1. fgr_run on the slice W[n_g0:n_g1, :] (bias and scale slices alike) with reduce =
- *      FGR_RED_MAX_SUMEXP (for a final LSE or MAX_SUMEXP), FGR_RED_MAXSUM (final MAXSUM) or
- *      FGR_RED_SOFTMAX with `out` given (final softmax) -> a local pair per row, [rows, 2] fp32;
+ *      FGR_RED_MAX_SUMEXP (for a final LSE or MAX_SUMEXP), FGR_RED_MAXSUM (final MAXSUM),
+ *      FGR_RED_MEANVAR (final MEANVAR) or FGR_RED_SOFTMAX with `out` given (final softmax) -> a local
+ *      pair per row, [rows, 2] fp32.  (MEANVAR needs the slice widths to weight the pairs: the slices must
+ *      be the contiguous partition of N in groups of 8 (bf16) / 4 (fp32) columns, in shard order, the first
+ *      (N / group) % G shards one group wider; n_total = N.)
  *   2. all-gather of the pairs (NCCL; rows * 8 bytes per GPU) -> pairs[G][rows][2] on every GPU;
  *   3. fgr_combine_shards merges the G pairs of every row in ascending shard order (so every GPU
  *      computes bit-identical results) and writes `out` as the unsharded operator would; for softmax
@@ -303,7 +306,7 @@ typedef struct fgr_shard_desc {
   int32_t shard;           /* this GPU's index in [0, G) (SOFTMAX only) */
   int32_t n_local;         /* columns of this GPU's slice (SOFTMAX only) */
   int32_t device;          /* CUDA device ordinal */
-  int32_t reserved;        /* 0 */
+  int32_t n_total;         /* MEANVAR only: N of the whole operator (the shard widths follow from it, see above) */
   int64_t rows;            /* batch * M */
   int64_t ldp;             /* row stride of P_local in elements; 0 = n_local */
 } fgr_shard_desc;

@@ -50,7 +50,7 @@ class fgr_reduce_desc(ctypes.Structure):
 class fgr_shard_desc(ctypes.Structure):
     _fields_ = [("struct_bytes", ctypes.c_uint32), ("shards", ctypes.c_int32), ("reduce", ctypes.c_int32),
                 ("dtype", ctypes.c_int32), ("shard", ctypes.c_int32), ("n_local", ctypes.c_int32),
-                ("device", ctypes.c_int32), ("reserved", ctypes.c_int32), ("rows", ctypes.c_int64),
+                ("device", ctypes.c_int32), ("n_total", ctypes.c_int32), ("rows", ctypes.c_int64),
                 ("ldp", ctypes.c_int64)]
 
 
@@ -193,10 +193,10 @@ def fgr_reduce_rows(M, N, dtype, reduce, A, P, out, *, lda=0, ldp=0, device=0, s
 
 
 def fgr_combine_shards(rows, shards, reduce, pairs, out, P_local=None, *, dtype=FGR_BF16, shard=0, n_local=0, ldp=0,
-                       device=0, stream=None, check=True) -> int:
+                       device=0, stream=None, check=True, n_total=0) -> int:
     """Merges the all-gathered per-shard row statistics ``pairs`` [shards, rows, 2] of an N-sharded
     operator (device pointers: ints or tensors); softmax also rescales the local slice ``P_local``."""
-    d = fgr_shard_desc(ctypes.sizeof(fgr_shard_desc), shards, reduce, dtype, shard, n_local, device, 0, rows, ldp)
+    d = fgr_shard_desc(ctypes.sizeof(fgr_shard_desc), shards, reduce, dtype, shard, n_local, device, n_total, rows, ldp)
     rc = lib().fgr_combine_shards(ctypes.byref(d), _addr(pairs), _addr(out), _addr(P_local), stream)
     if check and rc != FGR_OK:
         raise FgrError(rc, "fgr_combine_shards")

@@ -19,6 +19,7 @@ namespace {
 struct ShardParams {
   long long rows;
   int shards, reduce, shard, n_local;
+  int groups, align;     // MEANVAR: N / align column groups dealt to the shards, the first groups % shards get one more
   long long ldp;
   const float2* pairs;   // [shards][rows]
   float* out;
@@ -35,6 +36,21 @@ __device__ __forceinline__ void merge_exp(float& a, float& b, float2 v) {
 __global__ void __launch_bounds__(256) combine_rows_kernel(const ShardParams p) {
   const long long row = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (row >= p.rows) return;
+  if (p.reduce == FGR_RED_MEANVAR) {
+    // pairs are (mean, population variance) of a shard's columns; the shard widths follow the partition rule
+    const int base = p.groups / p.shards, extra = p.groups % p.shards;
+    float n = 0.0f, mean = 0.0f, m2 = 0.0f;
+    for (int g = 0; g < p.shards; ++g) {
+      const float nb = (float)((base + (g < extra ? 1 : 0)) * p.align);
+      const float2 v = p.pairs[(long long)g * p.rows + row];
+      const float tot = n + nb, delta = v.x - mean;
+      mean += delta * (nb / tot);
+      m2 += v.y * nb + delta * delta * (n * nb / tot);
+      n = tot;
+    }
+    reinterpret_cast<float2*>(p.out)[row] = make_float2(mean, m2 / n);
+    return;
+  }
   float a = -CUDART_INF_F, b = 0.0f;
   for (int g = 0; g < p.shards; ++g) {
     const float2 v = p.pairs[(long long)g * p.rows + row];
@@ -94,7 +110,18 @@ extern "C" int fgr_combine_shards(const fgr_shard_desc* d, const float* pairs, f
   using namespace fgr;
   if (!d || d->struct_bytes != sizeof(fgr_shard_desc) || !pairs) return FGR_ERR_INVALID_ARG;
   if (d->rows < 1 || d->shards < 1 || d->device < 0) return FGR_ERR_INVALID_ARG;
-  if (d->reduce < FGR_RED_LSE || d->reduce > FGR_RED_MAX_SUMEXP) return FGR_ERR_INVALID_ARG;
+  const bool meanvar = d->reduce == FGR_RED_MEANVAR;
+  if ((d->reduce < FGR_RED_LSE || d->reduce > FGR_RED_MAX_SUMEXP) && !meanvar) return FGR_ERR_INVALID_ARG;
+  int groups = 0, align = 0;
+  if (meanvar) {
+    // the column partition of the shards: n_total columns in groups of 8 (bf16) / 4 (fp32), contiguous slices in
+    // shard order, the first (groups % shards) shards one group wider
+    if (d->dtype != FGR_F32 && d->dtype != FGR_BF16) return FGR_ERR_INVALID_ARG;
+    align = d->dtype == FGR_F32 ? 4 : 8;
+    if (d->n_total < 1 || d->n_total % align) return FGR_ERR_INVALID_ARG;
+    groups = d->n_total / align;
+    if (groups < d->shards) return FGR_ERR_INVALID_ARG;
+  }
   if ((reinterpret_cast<uintptr_t>(pairs) & 7u) || (out && (reinterpret_cast<uintptr_t>(out) & 7u))) return FGR_ERR_INVALID_ARG;
   const bool softmax = d->reduce == FGR_RED_SOFTMAX;
   long long ldp = 0;
@@ -113,7 +140,7 @@ extern "C" int fgr_combine_shards(const fgr_shard_desc* d, const float* pairs, f
   int prev = -1;
   cudaGetDevice(&prev);
   if (prev != d->device && cudaSetDevice(d->device) != cudaSuccess) { cudaGetLastError(); return FGR_ERR_CUDA; }
-  ShardParams p = {d->rows, d->shards, d->reduce, d->shard, d->n_local, ldp, reinterpret_cast<const float2*>(pairs), out, P_local};
+  ShardParams p = {d->rows, d->shards, d->reduce, d->shard, d->n_local, groups, align, ldp, reinterpret_cast<const float2*>(pairs), out, P_local};
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   cudaError_t e;
   if (!softmax) {

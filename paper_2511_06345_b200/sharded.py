@@ -34,7 +34,7 @@ def local_reduce_kind(reduce: int) -> int:
     """The reduction each shard runs so that its row statistics can be merged into ``reduce``."""
     if reduce in (B.FGR_RED_LSE, B.FGR_RED_MAX_SUMEXP):
         return B.FGR_RED_MAX_SUMEXP
-    if reduce in (B.FGR_RED_MAXSUM, B.FGR_RED_SOFTMAX):
+    if reduce in (B.FGR_RED_MAXSUM, B.FGR_RED_SOFTMAX, B.FGR_RED_MEANVAR):
         return reduce
     raise ValueError("unknown reduction %r" % (reduce,))
 
@@ -65,6 +65,7 @@ class NShardedFusedGemmReduce:
         self.rank = rank if rank is not None else (dist.get_rank(group) if on else 0)
         self.reduce = reduce
         self.dtype = dtype
+        self.N = N
         self.n0, self.n1 = shard_range(N, self.world, self.rank, 8 if dtype == B.FGR_BF16 else 4)
         self.rows = batch * M
         self.device_index = device
@@ -82,7 +83,7 @@ class NShardedFusedGemmReduce:
                               device=self.local.device)
         stream = torch.cuda.current_stream(self.local.device).cuda_stream
         B.fgr_combine_shards(self.rows, self.world, self.reduce, gathered, out, Y if softmax else None, dtype=self.dtype,
-                             shard=self.rank, n_local=self.n1 - self.n0, device=self.device_index, stream=stream)
+                             shard=self.rank, n_local=self.n1 - self.n0, device=self.device_index, stream=stream, n_total=self.N)
         return Y, out
 
     def status(self) -> int:

@@ -74,6 +74,14 @@ def test_oracle_slices_merge_to_whole(world):
     mm, ss = _merge64(ms, False)
     np.testing.assert_allclose(mm, whole_ms[:, 0], rtol=0, atol=0)
     np.testing.assert_allclose(ss, whole_ms[:, 1], rtol=1e-12, atol=1e-12)
+    # (mean, variance): the slices' pairs weighted by the slice widths give the whole row's pair
+    mv = np.stack([_slice_problem(p, a, b, gi.RED_MEANVAR)[1] for a, b in edges])
+    widths = np.array([b - a for a, b in edges], dtype=np.float64)
+    _, whole_mv, _ = oracle.run_problem(gi_with(p, gi.RED_MEANVAR), want_y=False)
+    mean = (mv[:, :, 0] * widths[:, None]).sum(0) / p.N
+    var = ((mv[:, :, 1] + (mv[:, :, 0] - mean[None, :]) ** 2) * widths[:, None]).sum(0) / p.N
+    np.testing.assert_allclose(mean, whole_mv[:, 0], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(var, whole_mv[:, 1], rtol=1e-11)
     for g, (a, b) in enumerate(edges):
         P_loc = _slice_problem(p, a, b, gi.RED_SOFTMAX)[0]
         f = se[g, :, 1] * np.exp(se[g, :, 0] - m) / l
@@ -166,7 +174,7 @@ def _run_sharded_on_one_gpu(p, world, final):
     for g, (n0, n1) in enumerate(edges):
         st = torch.empty((rows, 2), dtype=torch.float32, device="cuda:0") if softmax else out
         fgr.fgr_combine_shards(rows, world, final, gathered, st, slices[g] if softmax else None, dtype=p.dtype, shard=g,
-                               n_local=n1 - n0, device=0)
+                               n_local=n1 - n0, device=0, n_total=p.N)
         stats.append(st)
         if not softmax:
             break                   # every shard would compute the same `out`
@@ -183,7 +191,7 @@ def _run_sharded_on_one_gpu(p, world, final):
 
 @pytest.mark.gpu
 @pytest.mark.parametrize("world", [1, 2, 3, 8])
-@pytest.mark.parametrize("final", [gi.RED_LSE, gi.RED_MAXSUM, gi.RED_MAX_SUMEXP, gi.RED_SOFTMAX])
+@pytest.mark.parametrize("final", [gi.RED_LSE, gi.RED_MAXSUM, gi.RED_MAX_SUMEXP, gi.RED_SOFTMAX, gi.RED_MEANVAR])
 def test_sharded_bf16_matches_oracle(cuda_device, world, final):
     from parity import compare
     # skinny, streaming-shaped problem with logits several units apart; ragged slices (N / 8 = 65 groups)
@@ -194,7 +202,7 @@ def test_sharded_bf16_matches_oracle(cuda_device, world, final):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("final", [gi.RED_LSE, gi.RED_SOFTMAX, gi.RED_MAXSUM])
+@pytest.mark.parametrize("final", [gi.RED_LSE, gi.RED_SOFTMAX, gi.RED_MAXSUM, gi.RED_MEANVAR])
 def test_sharded_fp32_matches_oracle(cuda_device, final):
     from parity import compare
     p = gi.make_config("c1", M=24, N=100, K=64, seed=2, scale_kind=gi.SCALE_SCALAR, scale=12.0, reduce=final)
