@@ -74,7 +74,7 @@ typedef enum { FGR_SCALE_NONE = 0, FGR_SCALE_SCALAR = 1, FGR_SCALE_PER_COLUMN = 
 typedef enum { FGR_RED_LSE = 0, FGR_RED_SOFTMAX = 1, FGR_RED_MAXSUM = 2, FGR_RED_MAX_SUMEXP = 3,
                /* (mean, population variance) of y over N: the row statistics of a normalisation layer.  Computed
                   per tile in two passes and merged pairwise (mean, sum of squared deviations), never as
-                  E[y^2] - E[y]^2.  Not on the FGR_PATH_SIMT_GEMV path. */
+                  E[y^2] - E[y]^2. */
                FGR_RED_MEANVAR = 6 } fgr_reduce;
 
 /* Execution paths (fgr_plan_info.path, fgr_desc.force_path). */

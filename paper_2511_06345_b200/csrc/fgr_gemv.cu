@@ -64,9 +64,13 @@ __global__ void __launch_bounds__(kGemvThreads, 1) gemv_kernel(const Params p, i
   const __nv_bfloat16* W = static_cast<const __nv_bfloat16*>(p.W) + (long long)bt * p.bsw;
   __nv_bfloat16* Y = static_cast<__nv_bfloat16*>(p.Y) + (long long)bt * p.bsy;
   const float* bias = p.bias ? p.bias + (p.bias_per_batch ? (long long)bt * p.N : 0) : nullptr;
-  const bool exp_kind = p.reduce != FGR_RED_MAXSUM;
+  const bool meanvar = p.reduce == FGR_RED_MEANVAR;
+  const bool exp_kind = p.reduce != FGR_RED_MAXSUM && !meanvar;
 
-  float s0 = -CUDART_INF_F, s1 = 0.0f;   // lane m < M: running (max, sum) or (max, sum of exp(y - max)) of row m
+  // lane m < M: running (max, sum) or (max, sum of exp(y - max)) of row m; for mean / variance the sums of
+  // (y - shift) and (y - shift)^2 against the first y this lane saw, and their count
+  float s0 = meanvar ? 0.0f : -CUDART_INF_F, s1 = 0.0f, shift = 0.0f;
+  int cnt = 0;
 
   for (int pass0 = n_begin; pass0 < n_end; pass0 += kGemvWarps * R) {
     const int n0 = pass0 + warp * R;
@@ -140,7 +144,13 @@ __global__ void __launch_bounds__(kGemvThreads, 1) gemv_kernel(const Params p, i
         float y = activation(p.act, z + (bias ? bias[n] : 0.0f)) * s;
         if (p.R) y += __bfloat162float(static_cast<const __nv_bfloat16*>(p.R)[(long long)bt * p.bsr + (long long)lane * p.ldr + n]);
         if (p.write_y) Y[(long long)lane * p.ldy + n] = __float2bfloat16_rn(y);
-        if (exp_kind) {
+        if (meanvar) {
+          if (cnt == 0) shift = y;
+          const float d = y - shift;
+          s0 += d;
+          s1 = fmaf(d, d, s1);
+          ++cnt;
+        } else if (exp_kind) {
           const float mn = fmaxf(s0, y);
           s1 = s1 * expf(s0 - mn) + expf(y - mn);
           s0 = mn;
@@ -151,6 +161,11 @@ __global__ void __launch_bounds__(kGemvThreads, 1) gemv_kernel(const Params p, i
       }
     }
   }
+  if (meanvar && cnt > 0) {   // -> (mean, sum of squared deviations) of this warp's columns of row `lane`
+    const float md = s0 / (float)cnt;
+    s1 = fmaxf(s1 - s0 * md, 0.0f);
+    s0 = shift + md;
+  }
 
   // combine the warps of this CTA in warp order (fixed, so results repeat bit for bit)
   __syncthreads();
@@ -158,9 +173,24 @@ __global__ void __launch_bounds__(kGemvThreads, 1) gemv_kernel(const Params p, i
   __syncthreads();
   if (warp == 0 && lane < p.M) {
     float a = -CUDART_INF_F, b = 0.0f;
+    float n = 0.0f;
+    if (meanvar) { a = 0.0f; }
     for (int w = 0; w < kGemvWarps; ++w) {
       const float2 v = red[w * MT + lane];
-      if (exp_kind) {
+      if (meanvar) {
+        // columns warp w finished: R per pass of kGemvWarps * R columns, clipped at the end of this CTA's range
+        int cw = 0;
+        for (int pass0 = n_begin; pass0 < n_end; pass0 += kGemvWarps * R) {
+          const int left = n_end - (pass0 + w * R);
+          cw += left <= 0 ? 0 : (left < R ? left : R);
+        }
+        if (cw > 0) {
+          const float nb = (float)cw, tot = n + nb, delta = v.x - a;
+          a += delta * (nb / tot);
+          b += v.y + delta * delta * (n * nb / tot);
+          n = tot;
+        }
+      } else if (exp_kind) {
         const float mn = fmaxf(a, v.x);
         if (mn > -CUDART_INF_F) b = b * expf(a - mn) + v.y * expf(v.x - mn);
         a = mn;

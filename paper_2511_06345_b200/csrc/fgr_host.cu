@@ -147,12 +147,11 @@ int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
     // fp32: CUDA-core FMA tiles, or for large compute-bound problems three tf32 tensor-core products
     // (the operand split costs one extra pass over X and W, so small or skinny problems stay on FMA)
     if (d.dtype == FGR_F32) path = (d.M >= 128 && d.N >= 128 && d.K >= 128 && pi.flop >= kTf32MinFlop) ? FGR_PATH_UMMA_TF32X3 : FGR_PATH_SIMT;
-    else if (d.M <= 4 && d.reduce != FGR_RED_SOFTMAX && d.reduce != FGR_RED_MEANVAR) path = FGR_PATH_SIMT_GEMV;   // a few GEMVs: CUDA cores keep up with HBM
+    else if (d.M <= 4 && d.reduce != FGR_RED_SOFTMAX) path = FGR_PATH_SIMT_GEMV;   // a few GEMVs: CUDA cores keep up with HBM
     else if (d.M <= 128 && pi.flop / pi.min_bytes < kRidgeFlopPerByte) path = FGR_PATH_UMMA_STREAM_W;
     else path = FGR_PATH_UMMA_TILED;
   }
-  if (path == FGR_PATH_SIMT_GEMV && (d.dtype != FGR_BF16 || d.M > 16 || d.reduce == FGR_RED_SOFTMAX || d.reduce == FGR_RED_MEANVAR))
-    return FGR_ERR_UNSUPPORTED;
+  if (path == FGR_PATH_SIMT_GEMV && (d.dtype != FGR_BF16 || d.M > 16 || d.reduce == FGR_RED_SOFTMAX)) return FGR_ERR_UNSUPPORTED;
   if ((path == FGR_PATH_UMMA_TILED || path == FGR_PATH_UMMA_STREAM_W) && d.dtype != FGR_BF16) return FGR_ERR_UNSUPPORTED;
   if (path == FGR_PATH_UMMA_TF32X3 && d.dtype != FGR_F32) return FGR_ERR_UNSUPPORTED;
   const bool tf32 = path == FGR_PATH_UMMA_TF32X3;

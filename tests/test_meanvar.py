@@ -9,9 +9,7 @@ import paper_2511_06345_b200 as fgr
 
 def test_plan_rules_for_meanvar():
     mk = lambda M, **kw: fgr.fgr_plan(fgr.make_desc(1, M, 2048, 512, fgr.FGR_BF16, 0, 0, fgr.FGR_RED_MEANVAR, **kw))
-    assert mk(2).path == fgr.FGR_PATH_UMMA_STREAM_W              # the skinny CUDA-core path has no mean / variance
-    with pytest.raises(fgr.FgrError):
-        mk(2, force_path=fgr.FGR_PATH_SIMT_GEMV)
+    assert mk(2).path == fgr.FGR_PATH_SIMT_GEMV and mk(8).path == fgr.FGR_PATH_UMMA_STREAM_W
     assert mk(512).path == fgr.FGR_PATH_UMMA_TILED
     with pytest.raises(fgr.FgrError):
         fgr.fgr_plan(fgr.make_desc(1, 8, 64, 64, fgr.FGR_BF16, 0, 0, 5))     # 4 and 5 belong to fgr_reduce_rows only
@@ -30,7 +28,9 @@ CASES = [
     (gi.DTYPE_BF16, 2, 257, 1000, 136, fgr.FGR_PATH_UMMA_TILED, 240, 1),
     (gi.DTYPE_BF16, 1, 129, 120, 512, fgr.FGR_PATH_UMMA_TILED, 64, 2),
     (gi.DTYPE_BF16, 1, 128, 2048, 320, fgr.FGR_PATH_UMMA_STREAM_W, 0, 0),
-    (gi.DTYPE_BF16, 1, 3, 2056, 128, fgr.FGR_PATH_AUTO, 0, 0),
+    (gi.DTYPE_BF16, 1, 3, 2056, 128, fgr.FGR_PATH_AUTO, 0, 0),             # the skinny CUDA-core path
+    (gi.DTYPE_BF16, 2, 11, 520, 72, fgr.FGR_PATH_SIMT_GEMV, 0, 0),
+    (gi.DTYPE_BF16, 1, 1, 8, 8, fgr.FGR_PATH_SIMT_GEMV, 0, 0),
     (gi.DTYPE_F32, 1, 300, 524, 200, fgr.FGR_PATH_UMMA_TF32X3, 0, 0),
     (gi.DTYPE_F32, 2, 129, 260, 36, fgr.FGR_PATH_UMMA_TF32X3, 64, 1),
 ]

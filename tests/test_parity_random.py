@@ -63,7 +63,7 @@ def _draw_extended(rng):
     C = int(rng.integers(1, 30)) * g
     K = max(taps, 1) * C
     red = int(rng.choice([0, 1, 2, 3, 6]))
-    if path == fgr.FGR_PATH_SIMT_GEMV and red in (gi.RED_SOFTMAX, gi.RED_MEANVAR):
+    if path == fgr.FGR_PATH_SIMT_GEMV and red == gi.RED_SOFTMAX:
         red = gi.RED_LSE
     kw = {}
     if path in (fgr.FGR_PATH_UMMA_TILED, fgr.FGR_PATH_UMMA_STREAM_W, fgr.FGR_PATH_UMMA_TF32X3):

@@ -32,7 +32,7 @@ CASES = [
 def test_residual_matches_oracle(cuda_device, case, red):
     from parity import compare, run_gpu
     dtype, B, M, N, K, path, tn, pair = case
-    if path == fgr.FGR_PATH_SIMT_GEMV and red in (gi.RED_SOFTMAX, gi.RED_MEANVAR):
+    if path == fgr.FGR_PATH_SIMT_GEMV and red == gi.RED_SOFTMAX:
         pytest.skip("not on the skinny CUDA-core path")
     for i, act in enumerate([gi.ACT_NONE, gi.ACT_GELU_TANH]):
         for wy in (0, 1):
