@@ -262,7 +262,7 @@ FGR_API int fgr_run_static(const fgr_desc* desc /*host*/, const void* X, const v
  * launch on `cuda_stream`, asynchronous, no workspace, no handle; bit-identical from run to run.
  * A row is reduced by a warp (short rows), a CTA, or - when there are fewer than about 300 rows and they
  * are long - by a thread-block cluster of 2, 4 or 8 CTAs whose per-CTA results are combined through
- * distributed shared memory (no scratch memory, still one launch).  MEANVAR rows always take one CTA.
+ * distributed shared memory (no scratch memory, still one launch).
  */
 enum { FGR_REDUCE_MAX = 4, FGR_REDUCE_SUM = 5 };   /* further values of `reduce` for fgr_reduce_rows only */
 typedef struct fgr_reduce_desc {

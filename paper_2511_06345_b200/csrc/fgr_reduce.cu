@@ -373,6 +373,77 @@ __global__ void __launch_bounds__(kThreads, 8) meanvar_rows_kernel(const ReduceP
   if (row_ok && sub == 0) reinterpret_cast<float2*>(p.out)[row] = make_float2(row_m.mean, row_m.m2 / (float)p.N);
 }
 
+// Mean / variance of few, long rows: the cluster form of the kernel above.  CTA r of a cluster of CL
+// reduces the r-th column segment to (count, mean, M2), stores the triple into slot r of the first
+// CTA's shared memory, and after the cluster barrier the first CTA folds the CL triples in rank order.
+__device__ __forceinline__ Moments fold(Moments a, Moments b) {
+  const float tot = a.n + b.n;
+  if (tot <= 0.0f) return a;
+  const float delta = b.mean - a.mean, wb = b.n / tot;
+  return {tot, fmaf(delta, wb, a.mean), a.m2 + b.m2 + delta * delta * (a.n * wb)};
+}
+template <typename T, int CL>
+__global__ void __launch_bounds__(kClusterThreads, 2) meanvar_rows_cluster_kernel(const ReduceParams p) {
+  constexpr int V = Vec<T>::kElems;
+  constexpr int G = kClusterThreads;
+  __shared__ Moments red[kClusterThreads / 32];
+  __shared__ Moments peers[CL];
+  const int rank = (int)(blockIdx.x % CL), lane = threadIdx.x & 31, sub = threadIdx.x;
+  const long long row = blockIdx.x / CL;
+  const T* a = static_cast<const T*>(p.A) + row * p.lda;
+  const int seg = ((p.N / V + CL - 1) / CL) * V;
+  const int c_lo = rank * seg < p.N ? rank * seg : p.N;
+  const int c_hi = c_lo + seg < p.N ? c_lo + seg : p.N;
+  Moments st = {0.0f, 0.0f, 0.0f};
+  if (c_lo + sub * V < c_hi) {
+    float shift = 0.0f, s1 = 0.0f, s2 = 0.0f;
+    int cnt = 0;
+    for (int c0 = c_lo + sub * V; c0 < c_hi; c0 += 4 * G * V) {
+      uint4 raw[4];
+      int nv = 0;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int c = c0 + u * G * V;
+        if (c < c_hi) { raw[u] = *reinterpret_cast<const uint4*>(a + c); nv = u + 1; }
+      }
+      if (cnt == 0) shift = __uint_as_float(sizeof(T) == 4 ? raw[0].x : raw[0].x << 16);
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (u < nv) {
+          float v[V];
+          Vec<T>::unpack(raw[u], v);
+#pragma unroll
+          for (int j = 0; j < V; ++j) { const float d = v[j] - shift; s1 += d; s2 = fmaf(d, d, s2); }
+        }
+      cnt += nv * V;
+    }
+    st.n = (float)cnt;
+    const float md = s1 / st.n;
+    st.mean = shift + md;
+    st.m2 = fmaxf(s2 - s1 * md, 0.0f);
+  }
+  const float cn = warp_sum(st.n), cs = warp_sum(st.n * st.mean);
+  const float wmean = cn > 0.0f ? cs / cn : 0.0f;
+  const float dm = st.mean - wmean;
+  const float q = warp_sum(fmaf(st.n * dm, dm, st.m2));
+  if (lane == 0) red[threadIdx.x >> 5] = {cn, wmean, q};
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    Moments m = red[0];
+#pragma unroll
+    for (int w = 1; w < kClusterThreads / 32; ++w) m = fold(m, red[w]);
+    store_remote(&peers[rank].n, 0u, m.n);
+    store_remote(&peers[rank].mean, 0u, m.mean);
+    store_remote(&peers[rank].m2, 0u, m.m2);
+  }
+  cluster_barrier();                                   // every thread of every CTA of the cluster
+  if (rank != 0 || threadIdx.x != 0) return;
+  Moments m = peers[0];
+#pragma unroll
+  for (int r = 1; r < CL; ++r) m = fold(m, peers[r]);
+  reinterpret_cast<float2*>(p.out)[row] = make_float2(m.mean, m.m2 / (float)p.N);
+}
+
 template <typename T>
 cudaError_t launch(const ReduceParams& p, cudaStream_t s) {
   const bool exp_kind = p.kind == FGR_RED_LSE || p.kind == FGR_RED_SOFTMAX || p.kind == FGR_RED_MAX_SUMEXP;
@@ -380,6 +451,10 @@ cudaError_t launch(const ReduceParams& p, cudaStream_t s) {
   const unsigned grid = warp_rows ? (unsigned)((p.M + kThreads / 32 - 1) / (kThreads / 32)) : (unsigned)p.M;
   const bool sum_kind = p.kind == FGR_RED_MAXSUM || p.kind == FGR_REDUCE_SUM;
   if (p.kind == FGR_RED_MEANVAR) {
+    const int mcl = cluster_size(p.M, p.N, Vec<T>::kElems);
+    if (mcl == 8) return launch_cluster(meanvar_rows_cluster_kernel<T, 8>, (unsigned)p.M * 8u, 8, p, s);
+    if (mcl == 4) return launch_cluster(meanvar_rows_cluster_kernel<T, 4>, (unsigned)p.M * 4u, 4, p, s);
+    if (mcl == 2) return launch_cluster(meanvar_rows_cluster_kernel<T, 2>, (unsigned)p.M * 2u, 2, p, s);
     if (warp_rows) meanvar_rows_kernel<T, 32><<<grid, kThreads, 0, s>>>(p);
     else meanvar_rows_kernel<T, kThreads><<<grid, kThreads, 0, s>>>(p);
     return cudaGetLastError();

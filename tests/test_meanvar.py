@@ -72,7 +72,8 @@ def test_meanvar_large_offset(cuda_device):
 
 @pytest.mark.gpu
 @pytest.mark.parametrize("dtype", [gi.DTYPE_F32, gi.DTYPE_BF16])
-@pytest.mark.parametrize("shape", [(1, 8), (5, 24), (300, 1000), (64, 2048), (9, 8200), (3, 40000)])
+@pytest.mark.parametrize("shape", [(1, 8), (5, 24), (300, 1000), (64, 2048), (9, 8200), (3, 40000),
+                                   (1, 1048576), (16, 262144), (5, 100008), (2, 33000)])   # the last four: a CTA cluster per row
 def test_reduce_rows_meanvar(cuda_device, dtype, shape):
     import torch
     import oracle
