@@ -18,3 +18,10 @@ def cuda_device():
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
     return torch.device("cuda:0")
+
+
+@pytest.fixture(scope="session", autouse=True)
+def built_library():
+    """libfgr.so is a build product (not in version control): compile it if it is missing or older than its sources."""
+    from paper_2511_06345_b200 import build as fgr_build
+    fgr_build.build()
