@@ -336,7 +336,7 @@ __global__ void __launch_bounds__(256) normalise_kernel(const Params p) {
           __nv_bfloat162 r = __floats2bfloat162_rn(__uint_as_float(w[j] << 16) * f, __uint_as_float(w[j] & 0xffff0000u) * f);
           w[j] = *reinterpret_cast<uint32_t*>(&r);
         }
-        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(y + c), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+        asm volatile("st.global.cs.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(y + c), "r"(w[0]), "r"(w[1]), "r"(w[2]),
                      "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
                      : "memory");
       }
