@@ -290,12 +290,38 @@ cudaError_t launch_cluster(Kernel kernel, unsigned grid, int cl, const ReducePar
   return cudaLaunchKernelEx(&cfg, kernel, p);
 }
 
+// Clusters of 16 CTAs are beyond the portable size: the kernel opts in, and the device is asked once (per
+// kernel) whether it can place such a cluster at all; if not, the caller falls back to 8.
+template <typename T>
+bool cluster16_available(void (*kernel)(ReduceParams)) {
+  static int state = 0;   // 0 = not asked yet, 1 = yes, -1 = no   (one instance per element type = per kernel)
+  if (state == 0) {
+    state = -1;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(16);
+      cfg.blockDim = dim3(kClusterThreads);
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = 16;
+      attr[0].val.clusterDim.y = 1;
+      attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) == cudaSuccess && n >= 1) state = 1;
+    }
+    cudaGetLastError();
+  }
+  return state == 1;
+}
+
 // Cluster size for a matrix of M rows of N elements of V per 16 bytes: 1 unless the rows are too few to
 // fill the machine (fewer than two per SM) and long enough to give every thread of a cluster's CTAs a
 // full iteration (four vectors) of the loop.
 int cluster_size(int M, int N, int V) {
   if (M >= 2 * 148) return 1;
-  for (int cl = 8; cl >= 2; cl >>= 1)   // 8 is the portable maximum (16, opt-in, measured: LSE 47 -> 39 us, max 26 -> 30 us)
+  for (int cl = 8; cl >= 2; cl >>= 1)   // 8 is the portable maximum
     if ((long long)N >= (long long)cl * kClusterThreads * V * 4 && (long long)M * cl <= 0x7fffffffLL) return cl;
   return 1;
 }
@@ -468,6 +494,11 @@ cudaError_t launch(const ReduceParams& p, cudaStream_t s) {
     if (sum_kind) return launch_cluster(reduce_rows_cluster_kernel<T, false, true, CLv>, cgrid, CLv, p, s); \
     return launch_cluster(reduce_rows_cluster_kernel<T, false, false, CLv>, cgrid, CLv, p, s); \
   } while (0)
+    // The exp kinds are bound by the arithmetic of the few SMs that hold a CTA: sixteen CTAs per row spread it
+    // over twice as many (measured on 16 x 4 Mi bf16: LSE 47 -> 39 us; the plain maximum got slower, 26 -> 30 us).
+    if (cl == 8 && exp_kind && (long long)p.N >= 16LL * kClusterThreads * Vec<T>::kElems * 4 && p.M * 16 <= 2 * 148 &&
+        cluster16_available<T>(reduce_rows_cluster_kernel<T, true, false, 16>))
+      return launch_cluster(reduce_rows_cluster_kernel<T, true, false, 16>, (unsigned)p.M * 16u, 16, p, s);
     if (cl == 8) FGR_CLUSTER_LAUNCH(8);
     if (cl == 4) FGR_CLUSTER_LAUNCH(4);
     FGR_CLUSTER_LAUNCH(2);
