@@ -5,6 +5,7 @@
 // (max, sum of 2^((v - max) log2 e)) pair and a plain sum, and a fixed shuffle / shared-memory tree
 // combines them, so results repeat bit for bit.
 #include <cuda_bf16.h>
+#include <mutex>
 #include <math_constants.h>
 
 #include "fgr.h"
@@ -12,6 +13,7 @@
 namespace {
 
 constexpr int kThreads = 256;
+constexpr int kMaxCluster = 16;         // 8 is the portable limit; larger clusters are asked for where they pay
 constexpr int kClusterThreads = 1024;   // CTAs of the cluster kernel: few CTAs, so each keeps many loads in flight
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -207,11 +209,17 @@ __device__ __forceinline__ void store_remote(const float* local, uint32_t cta, f
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(raddr) : "r"(laddr), "r"(cta));
   asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(raddr), "f"(v) : "memory");
 }
-template <typename T, bool EXP, bool SUM, int CL>
+__device__ __forceinline__ int cluster_ctas() {
+  uint32_t n;
+  asm("mov.u32 %0, %%cluster_nctaid.x;" : "=r"(n));
+  return (int)n;
+}
+template <typename T, bool EXP, bool SUM>
 __global__ void __launch_bounds__(kClusterThreads, 2) reduce_rows_cluster_kernel(const ReduceParams p) {
   constexpr int V = Vec<T>::kElems;
   __shared__ State red[kClusterThreads / 32];
-  __shared__ State peers[CL];
+  __shared__ State peers[kMaxCluster];
+  const int CL = cluster_ctas();                       // CTAs per row: any size from 1 to kMaxCluster
   const int rank = (int)(blockIdx.x % CL);            // = the CTA's rank in its cluster (cluster dims CL x 1 x 1)
   const long long row = blockIdx.x / CL;              // the grid is exactly M * CL CTAs
   const T* a = static_cast<const T*>(p.A) + row * p.lda;
@@ -244,10 +252,8 @@ __global__ void __launch_bounds__(kClusterThreads, 2) reduce_rows_cluster_kernel
   cluster_barrier();                                   // every thread of every CTA of the cluster
   if (!softmax && (rank != 0 || threadIdx.x != 0)) return;
   float m = peers[0].m;
-#pragma unroll
   for (int r = 1; r < CL; ++r) m = fmaxf(m, peers[r].m);
   float l = 0.0f, sum = 0.0f;
-#pragma unroll
   for (int r = 0; r < CL; ++r) {
     if (EXP) l += peers[r].m > -CUDART_INF_F ? peers[r].l * ex2((peers[r].m - m) * kLog2e) : 0.0f;
     sum += peers[r].s;
@@ -290,40 +296,62 @@ cudaError_t launch_cluster(Kernel kernel, unsigned grid, int cl, const ReducePar
   return cudaLaunchKernelEx(&cfg, kernel, p);
 }
 
-// Clusters of 16 CTAs are beyond the portable size: the kernel opts in, and the device is asked once (per
-// kernel) whether it can place such a cluster at all; if not, the caller falls back to 8.
-template <typename T>
-bool cluster16_available(void (*kernel)(ReduceParams)) {
-  static int state = 0;   // 0 = not asked yet, 1 = yes, -1 = no   (one instance per element type = per kernel)
-  if (state == 0) {
-    state = -1;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
-      cudaLaunchConfig_t cfg = {};
-      cfg.gridDim = dim3(16);
-      cfg.blockDim = dim3(kClusterThreads);
-      cudaLaunchAttribute attr[1];
-      attr[0].id = cudaLaunchAttributeClusterDimension;
-      attr[0].val.clusterDim.x = 16;
-      attr[0].val.clusterDim.y = 1;
-      attr[0].val.clusterDim.z = 1;
-      cfg.attrs = attr;
-      cfg.numAttrs = 1;
-      int n = 0;
-      if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) == cudaSuccess && n >= 1) state = 1;
+// How many clusters of cl CTAs of this kernel the device can hold at once (0 if it cannot place one).  Sizes
+// above 8 are beyond the portable limit: the kernel opts in first.  Asked once per kernel and size.
+int max_active_clusters(void (*kernel)(ReduceParams), int cl) {
+  struct Entry { void (*kernel)(ReduceParams); int n[kMaxCluster + 1]; };   // n: 0 = not asked yet, -1 = none
+  static Entry table[16] = {};
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
+  Entry* e = nullptr;
+  for (Entry& t : table) {
+    if (t.kernel == kernel || t.kernel == nullptr) { e = &t; break; }
+  }
+  if (!e || cl < 1 || cl > kMaxCluster) return 0;
+  if (e->kernel == nullptr) {
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+      cudaGetLastError();
+      return 0;
     }
+    e->kernel = kernel;
+  }
+  if (e->n[cl] == 0) {
+    e->n[cl] = -1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)cl);
+    cfg.blockDim = dim3(kClusterThreads);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cl;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) == cudaSuccess && n >= 1) e->n[cl] = n;
     cudaGetLastError();
   }
-  return state == 1;
+  return e->n[cl] > 0 ? e->n[cl] : 0;
 }
 
-// Cluster size for a matrix of M rows of N elements of V per 16 bytes: 1 unless the rows are too few to
-// fill the machine (fewer than two per SM) and long enough to give every thread of a cluster's CTAs a
-// full iteration (four vectors) of the loop.
-int cluster_size(int M, int N, int V) {
-  if (M >= 2 * 148) return 1;
-  for (int cl = 8; cl >= 2; cl >>= 1)   // 8 is the portable maximum
-    if ((long long)N >= (long long)cl * kClusterThreads * V * 4 && (long long)M * cl <= 0x7fffffffLL) return cl;
-  return 1;
+// Whether the cluster kernels (CTAs of 1024 threads, one or several per row) take a matrix of M rows of N
+// elements of V per 16 bytes: the rows are too few to fill the machine with a 256-thread CTA each (fewer
+// than two per SM) and long enough to give every thread of two such CTAs a full iteration (four vectors).
+bool few_long_rows(int M, int N, int V) {
+  return M < 2 * 148 && (long long)N >= 2LL * kClusterThreads * V * 4;
+}
+
+// CTAs per row for those kernels: as many as keep the grid at about 256 CTAs in one wave, every thread with
+// a full iteration, and all M clusters resident together.  Measured on 64 Mi bf16 elements in 1 to 295 rows
+// (LogSumExp and max + sum; the plain maximum is flat): the time falls with the cluster size up to exactly
+// these limits and jumps by 20 to 40 % past them; 8 CTAs per row throughout took up to 1.8 times as long
+// (256 rows), 16 wherever the device allows it up to 1.3 times (16 rows).
+int cluster_size(void (*kernel)(ReduceParams), int M, int N, int V) {
+  int cl = 256 / M < kMaxCluster ? 256 / M : kMaxCluster;
+  if (cl < 1) cl = 1;
+  while (cl > 2 && (long long)N < (long long)cl * kClusterThreads * V * 4) --cl;
+  while (cl > 8 && max_active_clusters(kernel, cl) < M) --cl;   // 8 is the portable limit, always placeable
+  return cl;
 }
 
 // (mean, population variance) of every row.  Each thread accumulates sum (v - c) and sum (v - c)^2
@@ -408,12 +436,13 @@ __device__ __forceinline__ Moments fold(Moments a, Moments b) {
   const float delta = b.mean - a.mean, wb = b.n / tot;
   return {tot, fmaf(delta, wb, a.mean), a.m2 + b.m2 + delta * delta * (a.n * wb)};
 }
-template <typename T, int CL>
+template <typename T>
 __global__ void __launch_bounds__(kClusterThreads, 2) meanvar_rows_cluster_kernel(const ReduceParams p) {
   constexpr int V = Vec<T>::kElems;
   constexpr int G = kClusterThreads;
   __shared__ Moments red[kClusterThreads / 32];
-  __shared__ Moments peers[CL];
+  __shared__ Moments peers[kMaxCluster];
+  const int CL = cluster_ctas();                       // CTAs per row: any size from 1 to kMaxCluster
   const int rank = (int)(blockIdx.x % CL), lane = threadIdx.x & 31, sub = threadIdx.x;
   const long long row = blockIdx.x / CL;
   const T* a = static_cast<const T*>(p.A) + row * p.lda;
@@ -465,7 +494,6 @@ __global__ void __launch_bounds__(kClusterThreads, 2) meanvar_rows_cluster_kerne
   cluster_barrier();                                   // every thread of every CTA of the cluster
   if (rank != 0 || threadIdx.x != 0) return;
   Moments m = peers[0];
-#pragma unroll
   for (int r = 1; r < CL; ++r) m = fold(m, peers[r]);
   reinterpret_cast<float2*>(p.out)[row] = make_float2(m.mean, m.m2 / (float)p.N);
 }
@@ -477,32 +505,20 @@ cudaError_t launch(const ReduceParams& p, cudaStream_t s) {
   const unsigned grid = warp_rows ? (unsigned)((p.M + kThreads / 32 - 1) / (kThreads / 32)) : (unsigned)p.M;
   const bool sum_kind = p.kind == FGR_RED_MAXSUM || p.kind == FGR_REDUCE_SUM;
   if (p.kind == FGR_RED_MEANVAR) {
-    const int mcl = cluster_size(p.M, p.N, Vec<T>::kElems);
-    if (mcl == 8) return launch_cluster(meanvar_rows_cluster_kernel<T, 8>, (unsigned)p.M * 8u, 8, p, s);
-    if (mcl == 4) return launch_cluster(meanvar_rows_cluster_kernel<T, 4>, (unsigned)p.M * 4u, 4, p, s);
-    if (mcl == 2) return launch_cluster(meanvar_rows_cluster_kernel<T, 2>, (unsigned)p.M * 2u, 2, p, s);
+    if (few_long_rows(p.M, p.N, Vec<T>::kElems)) {
+      const int mcl = cluster_size(meanvar_rows_cluster_kernel<T>, p.M, p.N, Vec<T>::kElems);
+      return launch_cluster(meanvar_rows_cluster_kernel<T>, (unsigned)p.M * (unsigned)mcl, mcl, p, s);
+    }
     if (warp_rows) meanvar_rows_kernel<T, 32><<<grid, kThreads, 0, s>>>(p);
     else meanvar_rows_kernel<T, kThreads><<<grid, kThreads, 0, s>>>(p);
     return cudaGetLastError();
   }
-  const int cl = cluster_size(p.M, p.N, Vec<T>::kElems);
-  if (cl > 1) {
-    const unsigned cgrid = (unsigned)p.M * (unsigned)cl;
-#define FGR_CLUSTER_LAUNCH(CLv) \
-  do { \
-    if (exp_kind) return launch_cluster(reduce_rows_cluster_kernel<T, true, false, CLv>, cgrid, CLv, p, s); \
-    if (sum_kind) return launch_cluster(reduce_rows_cluster_kernel<T, false, true, CLv>, cgrid, CLv, p, s); \
-    return launch_cluster(reduce_rows_cluster_kernel<T, false, false, CLv>, cgrid, CLv, p, s); \
-  } while (0)
-    // The exp kinds are bound by the arithmetic of the few SMs that hold a CTA: sixteen CTAs per row spread it
-    // over twice as many (measured on 16 x 4 Mi bf16: LSE 47 -> 39 us; the plain maximum got slower, 26 -> 30 us).
-    if (cl == 8 && exp_kind && (long long)p.N >= 16LL * kClusterThreads * Vec<T>::kElems * 4 && p.M * 16 <= 2 * 148 &&
-        cluster16_available<T>(reduce_rows_cluster_kernel<T, true, false, 16>))
-      return launch_cluster(reduce_rows_cluster_kernel<T, true, false, 16>, (unsigned)p.M * 16u, 16, p, s);
-    if (cl == 8) FGR_CLUSTER_LAUNCH(8);
-    if (cl == 4) FGR_CLUSTER_LAUNCH(4);
-    FGR_CLUSTER_LAUNCH(2);
-#undef FGR_CLUSTER_LAUNCH
+  if (few_long_rows(p.M, p.N, Vec<T>::kElems)) {
+    void (*kernel)(ReduceParams) = exp_kind   ? reduce_rows_cluster_kernel<T, true, false>
+                                   : sum_kind ? reduce_rows_cluster_kernel<T, false, true>
+                                              : reduce_rows_cluster_kernel<T, false, false>;
+    const int want = cluster_size(kernel, p.M, p.N, Vec<T>::kElems);
+    return launch_cluster(kernel, (unsigned)p.M * (unsigned)want, want, p, s);
   }
 #define FGR_REDUCE_LAUNCH(Gv) \
   do { \
