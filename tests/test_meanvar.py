@@ -73,7 +73,9 @@ def test_meanvar_large_offset(cuda_device):
 @pytest.mark.gpu
 @pytest.mark.parametrize("dtype", [gi.DTYPE_F32, gi.DTYPE_BF16])
 @pytest.mark.parametrize("shape", [(1, 8), (5, 24), (300, 1000), (64, 2048), (9, 8200), (3, 40000),
-                                   (1, 1048576), (16, 262144), (5, 100008), (2, 33000)])   # the last four: a CTA cluster per row
+                                   # from here on: clusters of 1 to 16 CTAs of 1024 threads per row
+                                   (1, 1048576), (16, 262144), (5, 100008), (2, 33000), (20, 400000), (7, 600008),
+                                   (100, 131072), (200, 70000)])
 def test_reduce_rows_meanvar(cuda_device, dtype, shape):
     import torch
     import oracle
