@@ -261,8 +261,8 @@ FGR_API int fgr_run_static(const fgr_desc* desc /*host*/, const void* X, const v
  * N, lda and ldp must be multiples of 8 (bf16) / 4 (fp32), else FGR_ERR_UNSUPPORTED.  One kernel
  * launch on `cuda_stream`, asynchronous, no workspace, no handle; bit-identical from run to run.
  * A row is reduced by a warp (short rows), a CTA, or - when there are fewer than about 300 rows and they
- * are long - by a thread-block cluster of 2, 4, 8 or (exponential kinds, where the device allows it) 16 CTAs
- * whose per-CTA results are combined through
+ * are long - by a thread-block cluster of 1 to 16 CTAs of 1024 threads (sizes above 8 where the device
+ * can hold all rows' clusters at once) whose per-CTA results are combined through
  * distributed shared memory (no scratch memory, still one launch).
  */
 enum { FGR_REDUCE_MAX = 4, FGR_REDUCE_SUM = 5 };   /* further values of `reduce` for fgr_reduce_rows only */
