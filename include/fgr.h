@@ -260,7 +260,7 @@ FGR_API int fgr_run_static(const fgr_desc* desc /*host*/, const void* X, const v
  *   out  device fp32: [M] (LSE, MAX, SUM) or [M, 2] (MAXSUM, MAX_SUMEXP, MEANVAR); required unless SOFTMAX
  * N, lda and ldp must be multiples of 8 (bf16) / 4 (fp32), else FGR_ERR_UNSUPPORTED.  One kernel
  * launch on `cuda_stream`, asynchronous, no workspace, no handle; bit-identical from run to run.
- * A row is reduced by a warp (short rows), a CTA, or - when there are fewer than about 300 rows and they
+ * A row is reduced by a warp (short rows), a CTA, or - when there are fewer than about 300 rows (softmax: 1024) and they
  * are long - by a thread-block cluster of 1 to 16 CTAs of 1024 threads (sizes above 8 where the device
  * can hold all rows' clusters at once) whose per-CTA results are combined through
  * distributed shared memory (no scratch memory, still one launch).

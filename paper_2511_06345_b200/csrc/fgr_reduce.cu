@@ -337,8 +337,11 @@ int max_active_clusters(void (*kernel)(ReduceParams), int cl) {
 // Whether the cluster kernels (CTAs of 1024 threads, one or several per row) take a matrix of M rows of N
 // elements of V per 16 bytes: the rows are too few to fill the machine with a 256-thread CTA each (fewer
 // than two per SM) and long enough to give every thread of two such CTAs a full iteration (four vectors).
-bool few_long_rows(int M, int N, int V) {
-  return M < 2 * 148 && (long long)N >= 2LL * kClusterThreads * V * 4;
+// Softmax, which walks its row twice, keeps the 1024-thread CTA (one per row) up to 1024 rows: on rows of
+// 64 Ki to 900 Ki bf16 elements it took 70 us against 114 at 296 rows, 69 against 82 at 560, 65 against 70
+// at 900, while the one-pass kinds are level with the 256-thread kernel from about 300 rows on.
+bool few_long_rows(int M, int N, int V, bool softmax) {
+  return M < (softmax ? 1024 : 2 * 148) && (long long)N >= 2LL * kClusterThreads * V * 4;
 }
 
 // CTAs per row for those kernels: as many as keep the grid at about 256 CTAs in one wave, every thread with
@@ -505,7 +508,7 @@ cudaError_t launch(const ReduceParams& p, cudaStream_t s) {
   const unsigned grid = warp_rows ? (unsigned)((p.M + kThreads / 32 - 1) / (kThreads / 32)) : (unsigned)p.M;
   const bool sum_kind = p.kind == FGR_RED_MAXSUM || p.kind == FGR_REDUCE_SUM;
   if (p.kind == FGR_RED_MEANVAR) {
-    if (few_long_rows(p.M, p.N, Vec<T>::kElems)) {
+    if (few_long_rows(p.M, p.N, Vec<T>::kElems, false)) {
       const int mcl = cluster_size(meanvar_rows_cluster_kernel<T>, p.M, p.N, Vec<T>::kElems);
       return launch_cluster(meanvar_rows_cluster_kernel<T>, (unsigned)p.M * (unsigned)mcl, mcl, p, s);
     }
@@ -513,7 +516,7 @@ cudaError_t launch(const ReduceParams& p, cudaStream_t s) {
     else meanvar_rows_kernel<T, kThreads><<<grid, kThreads, 0, s>>>(p);
     return cudaGetLastError();
   }
-  if (few_long_rows(p.M, p.N, Vec<T>::kElems)) {
+  if (few_long_rows(p.M, p.N, Vec<T>::kElems, p.kind == FGR_RED_SOFTMAX)) {
     void (*kernel)(ReduceParams) = exp_kind   ? reduce_rows_cluster_kernel<T, true, false>
                                    : sum_kind ? reduce_rows_cluster_kernel<T, false, true>
                                               : reduce_rows_cluster_kernel<T, false, false>;

@@ -96,10 +96,10 @@ def test_reduce_rows_deterministic_and_argument_checks(cuda_device):
 @pytest.mark.parametrize("dtype", [gi.DTYPE_F32, gi.DTYPE_BF16])
 @pytest.mark.parametrize("kind", KINDS)
 @pytest.mark.parametrize("shape", [(1, 1048576), (16, 262144), (5, 100008), (2, 33000), (40, 65536 + 8),
-                                   (20, 400000), (7, 600008), (100, 131072), (200, 70000)])
+                                   (20, 400000), (7, 600008), (100, 131072), (200, 70000), (300, 66000)])
 def test_reduce_rows_few_long_rows_cluster(cuda_device, dtype, kind, shape):
     """Few, long rows: a cluster of 1 to 16 CTAs of 1024 threads shares a row (16, 13, 12, 8, 6, 4, 3, 2 and 1
-    with these shapes) and the per-CTA states are combined through distributed shared memory (ragged
+    with these shapes; the last one takes this kernel for softmax only) and the per-CTA states are combined through distributed shared memory (ragged
     segments included)."""
     M, N = shape
     _check(_matrix(M, N, dtype, seed=60 + M, std=3.0), N, dtype, kind)
