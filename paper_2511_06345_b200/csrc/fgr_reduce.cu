@@ -267,15 +267,27 @@ __global__ void __launch_bounds__(kClusterThreads, 2) reduce_rows_cluster_kernel
     default: break;
   }
   if (softmax) {
-    // second pass over this CTA's own segment (read a moment ago: normally still in L2)
+    // second pass over this CTA's own segment, from its end to its start: what was read last is the most
+    // likely to be in L2 still (the matrix as a whole may exceed it); four vectors per iteration in flight
     T* dst = static_cast<T*>(p.P) + row * p.ldp;
     const float inv = 1.0f / l;
-    for (int c = c_lo + threadIdx.x * V; c < c_hi; c += kClusterThreads * V) {
-      float v[V];
-      Vec<T>::unpack(*reinterpret_cast<const uint4*>(a + c), v);
+    constexpr int kStep = kClusterThreads * V;
+    const int iters = (c_hi - c_lo + 4 * kStep - 1) / (4 * kStep);
+    for (int it = iters - 1; it >= 0; --it) {
+      const int c0 = c_lo + it * 4 * kStep + threadIdx.x * V;
+      uint4 raw[4];
 #pragma unroll
-      for (int j = 0; j < V; ++j) v[j] = ex2((v[j] - m) * kLog2e) * inv;
-      Vec<T>::store(dst + c, v);
+      for (int u = 0; u < 4; ++u)
+        if (c0 + u * kStep < c_hi) raw[u] = *reinterpret_cast<const uint4*>(a + c0 + u * kStep);
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (c0 + u * kStep < c_hi) {
+          float v[V];
+          Vec<T>::unpack(raw[u], v);
+#pragma unroll
+          for (int j = 0; j < V; ++j) v[j] = ex2((v[j] - m) * kLog2e) * inv;
+          Vec<T>::store(dst + c0 + u * kStep, v);
+        }
     }
   }
 }
