@@ -1,12 +1,18 @@
 #!/usr/bin/env python
 """Benchmark of the fused GEMM + epilogue + row-reduce operator on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config c2] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config all|c1..c5|...] [--impl ours|reference]
 
 One step = one pass of the whole hot path (GEMM mainloop, fused epilogue, per-tile row reduction,
 split-N merge / softmax normalisation) over one seeded synthetic problem of the named workload.
-Rank 0 prints ONE JSON line.  With N > 1 (torchrun) every rank runs its own problem on its own GPU
-(rows/batches are independent: no collective on the data path; weak scaling).
+Rank 0 prints ONE JSON line.  The default (--config all) times the five named workloads one after
+the other, W warm-up and K timed steps each: the top-level keys describe the largest one (c3) and
+"per_config" carries the record of every workload, "targets_met" the whole-step roofline fractions
+against the stated targets.  --config NAME times that workload alone.
+
+With N > 1 every rank runs its own problems on its own GPU (rows / batches are independent: no
+collective on the data path; weak scaling).  `python bench.py --gpus N` without a launcher starts
+the N ranks itself (torch.distributed.run on 127.0.0.1); under torchrun it uses the ranks it is given.
 
 Timing: W warm-up steps, then K steps between two CUDA events on the launching stream, bracketed
 by a barrier and a device synchronise; max over ranks.  Consecutive steps use different input and
@@ -59,7 +65,7 @@ def load_peaks():
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the GPU works."""
 
-    def __init__(self, index: int, period_s: float = 0.005):
+    def __init__(self, index: int, period_s: float = 0.001):
         self.index, self.period = index, period_s
         self.samples = []          # (host time, sm MHz, reasons bitmask)
         self.max_mhz = None
@@ -139,6 +145,53 @@ def dist_env():
     return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
 
 
+class Ctx:
+    """What every leg of the benchmark shares: the rank layout, the device, the process group, the peaks."""
+
+    def __init__(self, backend: str = "nccl", use_gpu: bool = True):
+        self.rank, self.local_rank, self.world = dist_env()
+        self.peaks, self.peak_src = load_peaks()
+        self.dev = None
+        if use_gpu:
+            import torch
+            if not torch.cuda.is_available():
+                raise SystemExit("bench.py needs a CUDA device: the operator has no CPU path")
+            torch.cuda.set_device(self.local_rank)
+            self.dev = torch.device("cuda", self.local_rank)
+        if self.world > 1:
+            import torch.distributed as dist
+            if backend == "nccl":
+                dist.init_process_group("nccl", device_id=self.dev)
+            else:
+                dist.init_process_group(backend)
+
+    def barrier(self):
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        if self.dev is not None:
+            import torch
+            torch.cuda.synchronize(self.dev)
+
+    def close(self):
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+def launch_ranks(n: int) -> int:
+    """`python bench.py --gpus N` without a launcher: start N local ranks of this same command line
+    (one per GPU, rendezvous on 127.0.0.1) and pass their output through."""
+    import socket
+    import subprocess
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def oracle_sample(p, seconds: float):
     """Times the CPU oracle, as it stands, on a leading block of rows sized for about `seconds`."""
     import numpy as np
@@ -164,14 +217,26 @@ def unit_and_value(cfg, p, seconds_per_step, n_problems=1):
     return "TFLOP/s", n_problems * p.flop / seconds_per_step / 1e12
 
 
+ACT_NAMES = ["none", "relu", "gelu_tanh", "sigmoid", "tanh", "silu"]
+SCALE_NAMES = ["none", "scalar", "per_column"]
+REDUCE_NAMES = {0: "lse", 1: "softmax", 2: "maxsum", 3: "max_sumexp", 6: "meanvar"}
+
+
+def shape_keys(cfg, p):
+    """The keys of `config` that name the workload itself (both arms print exactly these)."""
+    import fgr_inputs as gi
+    return {"workload": cfg, "batch": p.batch, "M": p.M, "N": p.N, "K": p.K, "act": ACT_NAMES[p.act],
+            "scale": SCALE_NAMES[p.scale_kind], "reduce": REDUCE_NAMES[p.reduce],
+            "write_y": int(bool(p.write_y) or p.reduce == gi.RED_SOFTMAX), "conv_taps": p.conv_taps, "w_shared": p.w_shared}
+
+
 def run_reference(args):
     rank, _, world = dist_env()
     if rank != 0:
         return
-    import fgr_inputs as gi
-    p = make_cfg(args.config, seed=0)
+    cfg = HEADLINE if args.config == "all" else args.config
+    p = make_cfg(cfg, seed=0)
     per_step = min(2.0, 60.0 / max(args.steps, 1))   # the whole run stays near a minute of CPU time
-    flop = dt = 0.0
     threads = rows = 0
     for _ in range(max(args.warmup, 0)):
         oracle_sample(p, 0.2)
@@ -180,37 +245,54 @@ def run_reference(args):
         flop, dt, threads, rows = oracle_sample(p, per_step)
         f_sum += flop
         t_sum += dt
-    if args.config in HBM_BOUND:
+    if cfg in HBM_BOUND:
         unit, value = "GB/s", (f_sum / p.flop) * p.min_bytes() / t_sum / 1e9
     else:
         unit, value = "TFLOP/s", f_sum / t_sum / 1e12
     sample = "%d of %d rows per step (every %d-th row), all N and K" % (rows, p.batch * p.M, max(1, p.batch * p.M // rows))
+    config = shape_keys(cfg, p)
+    config["note"] = "CPU fp64 oracle on a bounded row sample"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": unit, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * t_sum / max(args.steps, 1), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.config, "note": "CPU fp64 oracle on a bounded row sample"},
+        "config": config,
         "cpu_baseline": {"value": value, "unit": unit, "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
 
-def run_ours(args):
+HEADLINE = "c3"                                     # the largest of the five named workloads
+NAMED = ["c1", "c2", "c3", "c4", "c5"]
+TARGETS = {"c2": 0.60, "c3": 0.60, "c5": 0.60, "c4": 0.70}   # whole-step fraction of the measured peak
+
+
+def empty_launch_us(ctx, n: int = 200) -> float:
+    """Mean time of one launch of an empty kernel in a back-to-back stream of n: the floor under any
+    step that is bound by launch latency (c1)."""
+    import torch
+    import paper_2511_06345_b200 as fgr
+    stream = torch.cuda.current_stream(ctx.dev).cuda_stream
+    fgr.fgr_profile_empty_launches(16, ctx.local_rank, stream)
+    torch.cuda.synchronize(ctx.dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    fgr.fgr_profile_empty_launches(n, ctx.local_rank, stream)
+    e1.record()
+    torch.cuda.synchronize(ctx.dev)
+    return e0.elapsed_time(e1) * 1e3 / n
+
+
+def measure_fused(cfg, args, ctx, with_e2e=True, with_cpu=True):
+    """Times one workload of the fused operator; returns the record rank 0 prints (None elsewhere)."""
     import numpy as np
     import torch
     import fgr_inputs as gi
     import paper_2511_06345_b200 as fgr
 
-    rank, local_rank, world = dist_env()
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the operator has no CPU path")
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
-    cfg = args.config
-    peaks, peak_src = load_peaks()
+    rank, local_rank, world, dev = ctx.rank, ctx.local_rank, ctx.world, ctx.dev
+    peaks, peak_src = ctx.peaks, ctx.peak_src
+    warmup = max(args.warmup, 3)
 
     sampler = ClockSampler(local_rank)
     # ---- inputs: a rotation of distinct problems so that no step finds its operands in L2
@@ -256,16 +338,10 @@ def run_ours(args):
         s = sets[i % rot]
         fgr.fgr_run(h, s["X"], s["W"], s["bias"], s["scale"], s["Y"], s["out"], ws, ws_bytes, stream)
 
-    def barrier():
-        if world > 1:
-            import torch.distributed as dist
-            dist.barrier()
-        torch.cuda.synchronize(dev)
-
     sampler.start()
-    for i in range(max(args.warmup, 3)):
+    for i in range(warmup):
         step(i)
-    barrier()
+    ctx.barrier()
     # ---- the timed region: K steps, nothing else on the stream
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_host0 = time.perf_counter()
@@ -273,8 +349,7 @@ def run_ours(args):
     for i in range(args.steps):
         step(i)
     e1.record()
-    barrier()
-    t_host1 = time.perf_counter()
+    ctx.barrier()
     status = fgr.fgr_get_status(h)
     if status != fgr.FGR_OK:
         raise SystemExit("device status after the timed region: " + fgr.fgr_status_string(status))
@@ -285,7 +360,7 @@ def run_ours(args):
     fgr.fgr_profile_enable(h, True)
     for i in range(args.steps):
         step(i)
-    barrier()
+    ctx.barrier()
     t_host2 = time.perf_counter()
     sampler.stop()
     fgr.fgr_profile_enable(h, False)
@@ -308,21 +383,28 @@ def run_ours(args):
             roof["frac_of_sustained_peak"] = roof["achieved"] / (peaks["bf16_tflops_sustained"] * (1.1 / 2.25) / 3.0)
             roof["peak_note"] = "measured bf16 rate x 1.1/2.25 (nominal tf32 : bf16) / 3 products per fp32 product"
     roof["frac"] = roof["achieved"] / roof["peak"]
+    # the whole step (every launch of fgr_run, one GPU's share of the job) against the same peak
+    roof["step_frac"] = value / world / roof["peak"]
     roof["peak_source"] = peak_src + (" (burst)" if roof["bound"] == "tensor" else "")
     roof["kernel"] = {fgr.FGR_PATH_UMMA_TILED: "umma_kernel", fgr.FGR_PATH_UMMA_STREAM_W: "umma_kernel",
                       fgr.FGR_PATH_SIMT_GEMV: "gemv_kernel", fgr.FGR_PATH_UMMA_TF32X3: "umma_kernel (tf32)"}.get(plan.path, "simt_gemm_kernel")
     roof["kernel_us"] = kern_s * 1e6
     roof["timing"] = "CUDA events around each of %d launches of the kernel, in a second pass of the same steps" % kern_runs
     roof["traffic"] = TRAFFIC.get(cfg)
+    if cfg == "c1":
+        # launch-latency bound: the fractions above mean little; the floor is the cost of a launch
+        roof["note"] = "launch-latency bound (33.6 Mflop): compare the step with empty_launch_us x launches per step"
+        roof["empty_launch_us"] = empty_launch_us(ctx)
+        roof["launches_per_step"] = plan.launches
 
     # ---- end to end: host buffers through fgr_run_host, copies inside the timed region
     e2e = None
-    if not args.no_e2e:
+    if with_e2e:
         hp = {k: (None if v is None else v.cpu().pin_memory()) for k, v in sets[0].items()}
         e2e_steps = max(3, min(args.steps, 20))
         for _ in range(2):
             fgr.fgr_run_host(h, hp["X"], hp["W"], hp["bias"], hp["scale"], hp["Y"], hp["out"])
-        barrier()
+        ctx.barrier()
         t0 = time.perf_counter()
         for _ in range(e2e_steps):
             fgr.fgr_run_host(h, hp["X"], hp["W"], hp["bias"], hp["scale"], hp["Y"], hp["out"])
@@ -334,11 +416,14 @@ def run_ours(args):
         d2h = sum(hp[k].numel() * hp[k].element_size() for k in ("Y", "out") if hp[k] is not None)
         e2e = {"value": ev, "unit": eu, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                "ms_per_step": dt * 1e3}
+        del hp
     fgr.fgr_destroy(h)
+    del sets, ws
+    torch.cuda.empty_cache()
 
     # ---- the CPU oracle timed beside it (rank 0, single-GPU runs only)
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and with_cpu:
         flop, dt, threads, nrows = oracle_sample(p, 12.0)
         if cfg in HBM_BOUND:
             cu, cv = "GB/s", (flop / p.flop) * p.min_bytes() / dt / 1e9
@@ -347,28 +432,65 @@ def run_ours(args):
         cpu = {"value": cv, "unit": cu, "cores": threads, "kind": "oracle", "seconds": dt,
                "sample": "%d of %d rows (evenly spaced), all N and K, fp64 triple loop" % (nrows, rows)}
 
-    if rank == 0:
-        line = {
-            "metric": METRIC, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16" if b16 else ("tf32x3" if plan.path == fgr.FGR_PATH_UMMA_TF32X3 else "f32"), "data": "synthetic",
-            "config": {"workload": cfg, "batch": p.batch, "M": p.M, "N": p.N, "K": p.K,
-                       "act": ["none", "relu", "gelu_tanh"][p.act], "scale": ["none", "scalar", "per_column"][p.scale_kind],
-                       "reduce": {0: "lse", 1: "softmax", 2: "maxsum", 3: "max_sumexp", 6: "meanvar"}[p.reduce], "write_y": int(need_y),
-                       "conv_taps": p.conv_taps, "w_shared": p.w_shared,
-                       "path": fgr.fgr_path_name(plan.path), "tile": [plan.tile_m, plan.tile_n], "stages": plan.stages,
-                       "grid": plan.grid, "l2": "rotating %d distinct input/output sets (%.0f MB > 126 MB L2)" % (rot, rot * set_bytes / 1e6),
-                       "parallelism": "independent problems per GPU, no collective" if world > 1 else "1 GPU"},
-            "clocks": clocks, "gpu_launches": args.steps * plan.launches, "roofline": roof,
-        }
-        if e2e is not None:
-            line["e2e"] = e2e
-        if cpu is not None:
-            line["cpu_baseline"] = cpu
+    if rank != 0:
+        return None
+    config = shape_keys(cfg, p)
+    config.update({"path": fgr.fgr_path_name(plan.path), "tile": [plan.tile_m, plan.tile_n], "stages": plan.stages,
+                   "grid": plan.grid, "l2": "rotating %d distinct input/output sets (%.0f MB > 126 MB L2)" % (rot, rot * set_bytes / 1e6),
+                   "parallelism": "independent problems per GPU, no collective" if world > 1 else "1 GPU"})
+    line = {
+        "metric": METRIC, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if b16 else ("tf32x3" if plan.path == fgr.FGR_PATH_UMMA_TF32X3 else "f32"), "data": "synthetic",
+        "config": config, "clocks": clocks, "gpu_launches": args.steps * plan.launches, "roofline": roof,
+    }
+    if e2e is not None:
+        line["e2e"] = e2e
+    if cpu is not None:
+        line["cpu_baseline"] = cpu
+    return line
+
+
+def run_ours(args, ctx):
+    line = measure_fused(args.config, args, ctx, with_e2e=not args.no_e2e, with_cpu=not args.no_cpu_baseline)
+    if line is not None:
         print(json.dumps(line))
-    if world > 1:
-        import torch.distributed as dist
-        dist.destroy_process_group()
+
+
+def run_all(args, ctx):
+    """The default: every named workload, W warm-up + K timed steps each.  The top level of the line is
+    the record of the largest workload; per_config holds all five, trimmed to what differs."""
+    records = {}
+    for cfg in NAMED:
+        head = cfg == HEADLINE
+        records[cfg] = measure_fused(cfg, args, ctx, with_e2e=head and not args.no_e2e,
+                                     with_cpu=head and not args.no_cpu_baseline)
+    if ctx.rank != 0:
+        return
+    line = dict(records[HEADLINE])
+    per, met = {}, {}
+    for cfg in NAMED:
+        r = records[cfg]
+        per[cfg] = {k: r[k] for k in ("value", "unit", "ms_per_step", "dtype", "config", "clocks", "gpu_launches", "roofline")}
+        if cfg in TARGETS:
+            f = r["roofline"]["step_frac"]
+            met[cfg] = {"bound": r["roofline"]["bound"], "step_frac": f, "kernel_frac": r["roofline"]["frac"],
+                        "target": TARGETS[cfg], "met": bool(f >= TARGETS[cfg])}
+    line["per_config"] = per
+    line["targets_met"] = met
+    line["gpu_launches"] = sum(r["gpu_launches"] for r in records.values())
+    line["gpu_launches_note"] = "kernels launched inside the five timed regions together (the top-level workload alone: %d)" % records[HEADLINE]["gpu_launches"]
+    print(json.dumps(line))
+
+
+def run_plumbing(args, ctx):
+    """Rendezvous, barrier, the max over ranks and rank 0's line, with no GPU work: what the CPU tests of
+    the launcher run (gloo).  It measures nothing and says so."""
+    ms = max_over_ranks(1.0 + ctx.rank, ctx.world)
+    ctx.barrier()
+    if ctx.rank == 0:
+        print(json.dumps({"metric": METRIC, "value": None, "unit": None, "n_gpus": ctx.world, "steps": 0, "warmup": 0,
+                          "plumbing_only": True, "max_over_ranks_check": ms}))
 
 
 REDUCE_CONFIGS = {   # stand-alone row reduction of a bf16 matrix, the paper's GPU case-study category (Section 4.4.1)
@@ -382,21 +504,17 @@ REDUCE_CONFIGS = {   # stand-alone row reduction of a bf16 matrix, the paper's G
 }
 
 
-def run_reduce(args):
+def run_reduce(args, ctx):
     """Bench leg of fgr_reduce_rows: same JSON contract; one step = one launch over one matrix."""
     import numpy as np
     import torch
+    import torch.distributed as dist
     import fgr_inputs as gi
     import paper_2511_06345_b200 as fgr
-    rank, local_rank, world = dist_env()
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+    rank, local_rank, world, dev = ctx.rank, ctx.local_rank, ctx.world, ctx.dev
     c = REDUCE_CONFIGS[args.config]
     M, N, kind = c["M"], c["N"], c["kind"]
-    peaks, peak_src = load_peaks()
+    peaks, peak_src = ctx.peaks, ctx.peak_src
     rot = 3                                                    # 3 x 134 MB > 126 MB L2
     hosts = [gi.f32_to_bf16_bits(gi.normal(1000 * rank + r, 9, M * N, 2.0)).reshape(M, N) for r in range(rot)]
     mats = [torch.from_numpy(h).view(torch.int16).view(torch.bfloat16).to(dev) for h in hosts]
@@ -464,29 +582,23 @@ def run_reduce(args):
         if cpu:
             line["cpu_baseline"] = cpu
         print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
 
 
 NSHARD_CONFIGS = {"c4n": "c4"}   # the skinny workload with W's rows (N) sharded over the ranks: strong scaling
 
 
-def run_nshard(args):
+def run_nshard(args, ctx):
     """Bench leg of the N-sharded operator: every rank streams its slice of W, one all-gather of the
     per-row statistics (rows x 8 bytes per rank, NCCL), then fgr_combine_shards.  The problem is fixed
     as ranks are added (strong scaling); value = the whole problem's algorithmic bytes / step time."""
     import numpy as np
     import torch
+    import torch.distributed as dist
     import fgr_inputs as gi
     import paper_2511_06345_b200 as fgr
-    rank, local_rank, world = dist_env()
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+    rank, local_rank, world, dev = ctx.rank, ctx.local_rank, ctx.world, ctx.dev
     base = NSHARD_CONFIGS[args.config]
-    peaks, peak_src = load_peaks()
+    peaks, peak_src = ctx.peaks, ctx.peak_src
     shape = make_cfg(base, materialize=False)
     op = fgr.NShardedFusedGemmReduce(shape.batch, shape.M, shape.N, shape.K, shape.dtype, shape.act, shape.scale_kind,
                                      shape.reduce, scale=shape.scale, device=local_rank)
@@ -567,13 +679,11 @@ def run_nshard(args):
             "e2e": {"value": p.min_bytes() / dt / 1e9, "unit": "GB/s", "h2d_bytes_per_step": sum(t.numel() * t.element_size() for t in hp),
                     "d2h_bytes_per_step": res.numel() * 4, "steps": e2e_steps, "ms_per_step": dt * 1e3}}))
     op.close()
-    if world > 1:
-        dist.destroy_process_group()
 
 
 # DRAM bytes per launch of the main kernel from ncu (dram__bytes_read.sum + dram__bytes_write.sum), one
-# capture per workload of the kernel as it stands (profiles/umma_kernel_<workload>.md); a workload
-# without a capture of the current kernel reports null.
+# capture per workload of the kernel as it stands; a workload without a capture of the current kernel
+# reports null.
 TRAFFIC = {"c2": 89.34e6, "c3": 182.95e6, "c4": 274.46e6, "c5": 70.78e6, "g2": 271.83e6,
            "r_max": 138.23e6, "r_lse": 139.97e6, "r_softmax": 224.41e6, "r_meanvar": 138.14e6,
            "r_max_long": 138.70e6, "r_lse_long": 140.99e6, "f2": 769.50e6, "v2": 124.35e6}
@@ -585,24 +695,37 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5"] + sorted(EXTRA_CONFIGS) + sorted(REDUCE_CONFIGS) + sorted(NSHARD_CONFIGS))
+    ap.add_argument("--config", default="all", choices=["all"] + NAMED + sorted(EXTRA_CONFIGS) + sorted(REDUCE_CONFIGS) + sorted(NSHARD_CONFIGS))
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"], help="process-group backend of a multi-rank run")
+    ap.add_argument("--plumbing-only", action="store_true",
+                    help="start the ranks, meet, print rank 0's line and stop: no GPU work, no measurement")
     args = ap.parse_args()
-    if args.config in NSHARD_CONFIGS:
-        if args.impl == "reference":
+    if args.impl == "reference":
+        # the CPU oracle, on rank 0 alone; the other ranks of a multi-rank launch exit at once
+        if args.config in NSHARD_CONFIGS:
             args.config = NSHARD_CONFIGS[args.config]     # the oracle has no shards: the same workload, whole
-            run_reference(args)
-        else:
-            run_nshard(args)
-    elif args.config in REDUCE_CONFIGS:
-        if args.impl == "reference":
+        if args.config in REDUCE_CONFIGS:
             raise SystemExit("the reference arm covers the fused operator's workloads c1..c5")
-        run_reduce(args)
-    elif args.impl == "reference":
         run_reference(args)
-    else:
-        run_ours(args)
+        return
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1:
+        sys.exit(launch_ranks(args.gpus))
+    ctx = Ctx(backend=args.backend, use_gpu=not args.plumbing_only)
+    try:
+        if args.plumbing_only:
+            run_plumbing(args, ctx)
+        elif args.config == "all":
+            run_all(args, ctx)
+        elif args.config in NSHARD_CONFIGS:
+            run_nshard(args, ctx)
+        elif args.config in REDUCE_CONFIGS:
+            run_reduce(args, ctx)
+        else:
+            run_ours(args, ctx)
+    finally:
+        ctx.close()
 
 
 if __name__ == "__main__":

@@ -161,7 +161,11 @@ FGR_API int fgr_plan(const fgr_desc* desc /*host*/, int num_sms, fgr_plan_info* 
  */
 FGR_API int fgr_create(const fgr_desc* desc /*host*/, fgr_handle** out /*host, out*/);
 
-/* Bytes of device workspace fgr_run needs (>= 256; 0 if h is NULL).  Contents need no initialisation. */
+/* Bytes of device workspace fgr_run needs (>= 256; 0 if h is NULL).  Contents need no initialisation when a
+ * workspace address is first given to a handle: fgr_run clears the status word at its head then.  While the
+ * same handle keeps being given the same address, the first 256 bytes belong to the library: if other code
+ * has written there in between (a caching allocator that recycled the block), zero those 256 bytes before
+ * the next fgr_run, or fgr_get_status may report the leftover value as an error code. */
 FGR_API size_t fgr_workspace_bytes(const fgr_handle* h);
 
 /* Copies the plan of a handle into *info. */
@@ -228,15 +232,22 @@ FGR_API int fgr_get_status(fgr_handle* h);
  * workspace fgr_run asks for, and has no handle.  Here the split-N partial pairs live in a fixed
  * array of FGR_STATIC_SCRATCH_BYTES inside the library image (each GPU that loads the library holds
  * those bytes until the process exits); the caller passes only the descriptor, inputs and outputs.
- * The call allocates nothing on the device or through any library, and creates no handle.
+ * The call makes no allocation call (no cudaMalloc / cudaFree, no allocating library routine) and creates
+ * no handle.  One thing to plan for: the CUDA runtime loads a library's device code lazily, so it is the
+ * FIRST call on a device that makes the driver load the module holding the array and reserve its
+ * FGR_STATIC_SCRATCH_BYTES.  Make that first call at start-up, before the device's memory is handed
+ * to whoever owns it; a first call on a device that is already full fails with FGR_ERR_CUDA.  Later
+ * calls leave the device's free memory unchanged.
  *
  *   - Always uses the CUDA-core path (FGR_PATH_SIMT; force_path must be AUTO or SIMT), fp32 or bf16.
  *     Results are those of fgr_run on that path.
  *   - Size limit: batch * M * ceil(N / 64) * 8 bytes must fit in FGR_STATIC_SCRATCH_BYTES, else
  *     FGR_ERR_WORKSPACE is returned and nothing is launched.
- *   - X, W, bias, scale_vec, Y, out: device pointers with the meaning and alignment fgr_run requires.
+ *   - X, W, bias, scale_vec, Y, out: device pointers with the meaning and alignment fgr_run requires
+ *     (the same checks are applied).
  *   - The first call on a device looks up the device address of the scratch array and checks the
- *     architecture; make that first call outside any stream capture.  Later calls only launch.
+ *     architecture (under a lock: host threads may race to it); make that first call outside any
+ *     stream capture.  Later calls only launch.
  *   - All calls on a device share the one array.  It keeps whatever the previous call left, which is
  *     harmless: every pair the merge pass reads is written earlier in the same call, so nothing has
  *     to be cleared.  Two calls whose kernels may overlap on the GPU (different streams, no ordering
@@ -324,6 +335,15 @@ FGR_API int fgr_combine_shards(const fgr_shard_desc* desc /*host*/, const float*
  */
 FGR_API int fgr_profile_enable(fgr_handle* h, int enable);
 FGR_API int fgr_profile_read(fgr_handle* h, double* main_kernel_ms /*host, out*/, int* runs /*host, out*/);
+
+/*
+ * fgr_profile_empty_launches: enqueues n launches of a kernel that does nothing (one warp, no memory
+ * access) on `cuda_stream` of `device`, asynchronously.  Timed by the caller with events around the call,
+ * it gives the cost of a kernel launch in a back-to-back stream on this machine - the floor under a
+ * problem so small that launch latency bounds it (the timing protocol of Section 4.1, Metrics, reports
+ * such a problem's microseconds beside that floor rather than a roofline fraction).
+ */
+FGR_API int fgr_profile_empty_launches(int n, int device, void* cuda_stream);
 
 /* Frees the handle and any staging memory it owns.  NULL is a no-op. */
 FGR_API int fgr_destroy(fgr_handle* h);

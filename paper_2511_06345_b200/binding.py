@@ -25,7 +25,7 @@ FGR_PATH_UMMA_TF32X3 = 5
 FGR_STATIC_SCRATCH_BYTES = 4 << 20
 
 EXPORTS = ("fgr_plan", "fgr_create", "fgr_workspace_bytes", "fgr_get_plan", "fgr_run", "fgr_run_host", "fgr_run_static", "fgr_reduce_rows", "fgr_combine_shards", "fgr_set_residual",
-           "fgr_get_status", "fgr_profile_enable", "fgr_profile_read", "fgr_destroy", "fgr_status_string", "fgr_path_name")
+           "fgr_get_status", "fgr_profile_enable", "fgr_profile_read", "fgr_profile_empty_launches", "fgr_destroy", "fgr_status_string", "fgr_path_name")
 
 
 class fgr_desc(ctypes.Structure):
@@ -96,6 +96,7 @@ def lib() -> ctypes.CDLL:
         L.fgr_get_status.argtypes, L.fgr_get_status.restype = [vp], i
         L.fgr_profile_enable.argtypes, L.fgr_profile_enable.restype = [vp, i], i
         L.fgr_profile_read.argtypes, L.fgr_profile_read.restype = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i)], i
+        L.fgr_profile_empty_launches.argtypes, L.fgr_profile_empty_launches.restype = [i, i, vp], i
         L.fgr_destroy.argtypes, L.fgr_destroy.restype = [vp], i
         L.fgr_status_string.argtypes, L.fgr_status_string.restype = [i], ctypes.c_char_p
         L.fgr_path_name.argtypes, L.fgr_path_name.restype = [i], ctypes.c_char_p
@@ -226,6 +227,14 @@ def fgr_profile_read(h):
     if rc != FGR_OK:
         raise FgrError(rc, "fgr_profile_read")
     return ms.value, n.value
+
+
+def fgr_profile_empty_launches(n: int, device: int = 0, stream=None) -> int:
+    """Enqueues n launches of a do-nothing kernel (the caller times them: the launch-latency floor)."""
+    rc = int(lib().fgr_profile_empty_launches(int(n), int(device), stream))
+    if rc != FGR_OK:
+        raise FgrError(rc, "fgr_profile_empty_launches")
+    return rc
 
 
 def fgr_destroy(h) -> int:

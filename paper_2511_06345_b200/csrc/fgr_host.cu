@@ -13,15 +13,39 @@
 
 using namespace fgr;
 
+namespace {
+constexpr int kMapSlots = 8;
+struct MapCache {
+  const void* key[kMapSlots];
+  CUtensorMap map[kMapSlots];
+  int next;                  // slot the next new pointer replaces (round robin)
+  const CUtensorMap* find(const void* ptr) const {
+    for (int i = 0; i < kMapSlots; ++i)
+      if (key[i] == ptr && ptr) return &map[i];
+    return nullptr;
+  }
+  CUtensorMap* claim(const void* ptr) {
+    const int i = next;
+    next = (next + 1) % kMapSlots;
+    key[i] = ptr;
+    return &map[i];
+  }
+  void forget(const void* ptr) {
+    for (int i = 0; i < kMapSlots; ++i)
+      if (key[i] == ptr) key[i] = nullptr;
+  }
+  void clear() { for (int i = 0; i < kMapSlots; ++i) key[i] = nullptr; }
+};
+}  // namespace
+
 struct fgr_handle {
   fgr_desc desc;
   fgr_plan_info plan;
   Params base;               // everything but the per-run pointers
   int num_sms;
-  // cached TMA descriptors (tcgen05 paths)
-  CUtensorMap tmap_x, tmap_w;
-  const void* cached_x;
-  const void* cached_w;
+  // cached TMA descriptors (tcgen05 paths): the last kMapSlots distinct base pointers per operand, so a
+  // caller that alternates between a few buffers (double buffering, a rotation) encodes each map once
+  MapCache maps_x, maps_w;
   // optional residual tensor (fgr_set_residual)
   const void* residual;
   long long ldr, bsr;
@@ -312,6 +336,8 @@ int encode_operand(CUtensorMap* map, const void* ptr, int K, int rows, int batch
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+__global__ void empty_kernel() {}
+
 }  // namespace
 
 extern "C" {
@@ -424,24 +450,37 @@ int fgr_run(fgr_handle* h, const void* X, const void* W, const float* bias, cons
     } else if (h->plan.path == FGR_PATH_SIMT_GEMV) {
       e = launch_gemv(p, p.tiles_n, p.tile_n, stream);
     } else if (tf32) {
-      // the tensor-core kernel reads the planes
-      if (workspace != h->cached_x) {   // the tensor maps describe the planes, which live in the workspace
+      // the tensor-core kernel reads the planes, which live in the workspace: both maps are keyed by it
+      const CUtensorMap* mx = h->maps_x.find(workspace);
+      const CUtensorMap* mw = h->maps_w.find(workspace);
+      if (!mx || !mw) {
         const long long ldp = 2LL * p.k_plane;
-        rc = encode_operand(&h->tmap_x, xp, (int)ldp, d.M, d.batch, ldp, (long long)d.M * ldp, kUmmaTileM, true);
-        if (rc == FGR_OK) rc = encode_operand(&h->tmap_w, wp, (int)ldp, d.N, d.w_shared ? 1 : d.batch, ldp, (long long)d.N * ldp, p.tile_n / p.cta_pair, true);
-        h->cached_x = rc == FGR_OK ? workspace : nullptr;
+        h->maps_x.forget(workspace);
+        h->maps_w.forget(workspace);
+        CUtensorMap* nx = h->maps_x.claim(workspace);
+        CUtensorMap* nw = h->maps_w.claim(workspace);
+        rc = encode_operand(nx, xp, (int)ldp, d.M, d.batch, ldp, (long long)d.M * ldp, kUmmaTileM, true);
+        if (rc == FGR_OK) rc = encode_operand(nw, wp, (int)ldp, d.N, d.w_shared ? 1 : d.batch, ldp, (long long)d.N * ldp, p.tile_n / p.cta_pair, true);
+        if (rc != FGR_OK) { h->maps_x.forget(workspace); h->maps_w.forget(workspace); }
+        mx = nx; mw = nw;
       }
-      if (rc == FGR_OK && e == cudaSuccess) e = launch_umma(p, &h->tmap_x, &h->tmap_w, h->plan.grid, h->plan.smem_bytes, stream);
+      if (rc == FGR_OK && e == cudaSuccess) e = launch_umma(p, mx, mw, h->plan.grid, h->plan.smem_bytes, stream);
     } else {
-      if (X != h->cached_x) {
-        rc = encode_operand(&h->tmap_x, X, d.K, d.M, d.batch, p.ldx, p.bsx, kUmmaTileM);
-        h->cached_x = rc == FGR_OK ? X : nullptr;
+      const CUtensorMap* mx = h->maps_x.find(X);
+      if (!mx) {
+        CUtensorMap* nx = h->maps_x.claim(X);
+        rc = encode_operand(nx, X, d.K, d.M, d.batch, p.ldx, p.bsx, kUmmaTileM);
+        if (rc != FGR_OK) h->maps_x.forget(X);
+        mx = nx;
       }
-      if (rc == FGR_OK && W != h->cached_w) {
-        rc = encode_operand(&h->tmap_w, W, d.K, d.N, d.w_shared ? 1 : d.batch, p.ldw, p.bsw, p.tile_n / p.cta_pair);
-        h->cached_w = rc == FGR_OK ? W : nullptr;
+      const CUtensorMap* mw = rc == FGR_OK ? h->maps_w.find(W) : nullptr;
+      if (rc == FGR_OK && !mw) {
+        CUtensorMap* nw = h->maps_w.claim(W);
+        rc = encode_operand(nw, W, d.K, d.N, d.w_shared ? 1 : d.batch, p.ldw, p.bsw, p.tile_n / p.cta_pair);
+        if (rc != FGR_OK) h->maps_w.forget(W);
+        mw = nw;
       }
-      if (rc == FGR_OK) e = launch_umma(p, &h->tmap_x, &h->tmap_w, h->plan.grid, h->plan.smem_bytes, stream);
+      if (rc == FGR_OK) e = launch_umma(p, mx, mw, h->plan.grid, h->plan.smem_bytes, stream);
     }
   }
   if (rc == FGR_OK && e == cudaSuccess && ev1) {
@@ -521,8 +560,8 @@ int fgr_run_host(fgr_handle* h, const void* X, const void* W, const float* bias,
       h->stage_bytes[i] = 0;
       if (cudaMalloc(&h->stage[i], want[i]) != cudaSuccess) rc = FGR_ERR_CUDA;
       else h->stage_bytes[i] = want[i];
-      if (i == 0) h->cached_x = nullptr;   // a new allocation may reuse an old address with other strides
-      if (i == 1) h->cached_w = nullptr;
+      if (i == 0) h->maps_x.clear();   // (the maps are keyed by address; a handle's strides never change, so a
+      if (i == 1) h->maps_w.clear();   //  reused address would still be described correctly: this is tidiness)
     }
   }
   cudaStream_t s = h->host_stream;
@@ -568,6 +607,20 @@ int fgr_profile_read(fgr_handle* h, double* main_kernel_ms, int* runs) {
   *main_kernel_ms = sum;
   *runs = n;
   return rc;
+}
+
+int fgr_profile_empty_launches(int n, int device, void* cuda_stream) {
+  if (n < 0 || device < 0) return FGR_ERR_INVALID_ARG;
+  int prev = -1;
+  cudaGetDevice(&prev);
+  if (prev != device && cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return FGR_ERR_CUDA; }
+  cudaError_t e = cudaSuccess;
+  for (int i = 0; i < n && e == cudaSuccess; ++i) {
+    empty_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>();
+    e = cudaGetLastError();
+  }
+  if (prev != device && prev >= 0) cudaSetDevice(prev);
+  return e == cudaSuccess ? FGR_OK : FGR_ERR_CUDA;
 }
 
 int fgr_destroy(fgr_handle* h) {

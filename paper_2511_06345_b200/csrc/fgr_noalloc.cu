@@ -14,6 +14,7 @@
 #include <cuda_runtime.h>
 
 #include <cstring>
+#include <mutex>
 
 #include "fgr_internal.h"
 
@@ -26,6 +27,7 @@ static __device__ __align__(256) unsigned char g_scratch[kScratchBytes];
 
 // Device address of g_scratch per device ordinal; filled by the first call on that device.
 float* g_scratch_addr[kMaxDevices] = {};
+std::mutex g_setup_mutex;
 
 }  // namespace
 
@@ -34,6 +36,8 @@ extern "C" {
 int fgr_run_static(const fgr_desc* desc, const void* X, const void* W, const float* bias, const float* scale_vec,
                    void* Y, float* out, void* cuda_stream) {
   if (!desc || !X || !W) return FGR_ERR_INVALID_ARG;
+  // the size field first: a shorter struct from an older caller must not be read past its end
+  if (desc->struct_bytes != sizeof(fgr_desc)) return FGR_ERR_INVALID_ARG;
   if (desc->force_path != FGR_PATH_AUTO && desc->force_path != FGR_PATH_SIMT) return FGR_ERR_UNSUPPORTED;
   if (desc->device < 0 || desc->device >= kMaxDevices) return FGR_ERR_INVALID_ARG;
   // validation and tiling come from the public planner, with the CUDA-core path selected
@@ -48,7 +52,8 @@ int fgr_run_static(const fgr_desc* desc, const void* X, const void* W, const flo
 
   const bool softmax = d.reduce == FGR_RED_SOFTMAX;
   if ((reinterpret_cast<uintptr_t>(X) & 15u) || (reinterpret_cast<uintptr_t>(W) & 15u) ||
-      (Y && (reinterpret_cast<uintptr_t>(Y) & 15u)) || (out && (reinterpret_cast<uintptr_t>(out) & 7u)))
+      (Y && (reinterpret_cast<uintptr_t>(Y) & 15u)) || (out && (reinterpret_cast<uintptr_t>(out) & 7u)) ||
+      (bias && (reinterpret_cast<uintptr_t>(bias) & 3u)) || (scale_vec && (reinterpret_cast<uintptr_t>(scale_vec) & 3u)))
     return FGR_ERR_INVALID_ARG;
   if ((d.write_y || softmax) && !Y) return FGR_ERR_INVALID_ARG;
   if (!softmax && !out) return FGR_ERR_INVALID_ARG;
@@ -58,14 +63,21 @@ int fgr_run_static(const fgr_desc* desc, const void* X, const void* W, const flo
   cudaGetDevice(&prev);
   if (prev != d.device && cudaSetDevice(d.device) != cudaSuccess) { cudaGetLastError(); return FGR_ERR_CUDA; }
   rc = FGR_OK;
-  if (!g_scratch_addr[d.device]) {
-    // one-time set-up on this device: architecture check and the device address of the scratch array
-    int major = 0;
-    void* addr = nullptr;
-    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, d.device) != cudaSuccess) rc = FGR_ERR_CUDA;
-    else if (major != 10) rc = FGR_ERR_ARCH;
-    else if (cudaGetSymbolAddress(&addr, g_scratch) != cudaSuccess || !addr) rc = FGR_ERR_CUDA;
-    else g_scratch_addr[d.device] = static_cast<float*>(addr);
+  float* scratch = nullptr;
+  {
+    // one-time set-up on this device (two host threads may make their first call together): architecture
+    // check and the device address of the scratch array.  With the CUDA runtime's lazy module loading this
+    // look-up is also what loads the module that holds the array, i.e. when the device reserves its bytes.
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    if (!g_scratch_addr[d.device]) {
+      int major = 0;
+      void* addr = nullptr;
+      if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, d.device) != cudaSuccess) rc = FGR_ERR_CUDA;
+      else if (major != 10) rc = FGR_ERR_ARCH;
+      else if (cudaGetSymbolAddress(&addr, g_scratch) != cudaSuccess || !addr) { cudaGetLastError(); rc = FGR_ERR_CUDA; }
+      else g_scratch_addr[d.device] = static_cast<float*>(addr);
+    }
+    scratch = g_scratch_addr[d.device];
   }
   if (rc == FGR_OK) {
     fgr::Params p;
@@ -81,7 +93,7 @@ int fgr_run_static(const fgr_desc* desc, const void* X, const void* W, const flo
     p.w_shared = d.w_shared;
     p.bsy = d.bsy ? d.bsy : (long long)d.M * p.ldy;
     p.X = X; p.W = W; p.bias = bias; p.scale_vec = scale_vec; p.Y = Y; p.out = out;
-    p.parts = g_scratch_addr[d.device];   // every pair the second kernel reads is written by the first
+    p.parts = scratch;   // every pair the second kernel reads is written by the first
     p.status = nullptr;                   // the CUDA-core kernels have no waits and report no status
     p.tile_n = plan.tile_n;
     p.half_n = plan.tile_n;

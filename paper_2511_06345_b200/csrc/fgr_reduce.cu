@@ -5,7 +5,9 @@
 // (max, sum of 2^((v - max) log2 e)) pair and a plain sum, and a fixed shuffle / shared-memory tree
 // combines them, so results repeat bit for bit.
 #include <cuda_bf16.h>
+#include <map>
 #include <mutex>
+#include <utility>
 #include <math_constants.h>
 
 #include "fgr.h"
@@ -308,27 +310,28 @@ cudaError_t launch_cluster(Kernel kernel, unsigned grid, int cl, const ReducePar
   return cudaLaunchKernelEx(&cfg, kernel, p);
 }
 
-// How many clusters of cl CTAs of this kernel the device can hold at once (0 if it cannot place one).  Sizes
-// above 8 are beyond the portable limit: the kernel opts in first.  Asked once per kernel and size.
+// How many clusters of cl CTAs of this kernel the current device can hold at once (0 if it cannot place
+// one).  Sizes above 8 are beyond the portable limit: the kernel opts in first.  Both the opt-in and the
+// occupancy answer belong to one device, so they are asked once per (device, kernel) and size, with that
+// device current (the caller has made it so).
 int max_active_clusters(void (*kernel)(ReduceParams), int cl) {
-  struct Entry { void (*kernel)(ReduceParams); int n[kMaxCluster + 1]; };   // n: 0 = not asked yet, -1 = none
-  static Entry table[16] = {};
+  struct Entry { bool opted_in; int n[kMaxCluster + 1]; };   // n: 0 = not asked yet, -1 = none
+  static std::map<std::pair<int, void (*)(ReduceParams)>, Entry> table;
   static std::mutex mu;
+  if (cl < 1 || cl > kMaxCluster) return 0;
+  int device = -1;
+  if (cudaGetDevice(&device) != cudaSuccess) { cudaGetLastError(); return 0; }
   std::lock_guard<std::mutex> lock(mu);
-  Entry* e = nullptr;
-  for (Entry& t : table) {
-    if (t.kernel == kernel || t.kernel == nullptr) { e = &t; break; }
-  }
-  if (!e || cl < 1 || cl > kMaxCluster) return 0;
-  if (e->kernel == nullptr) {
+  Entry& e = table[std::make_pair(device, kernel)];            // value-initialised on first use
+  if (!e.opted_in) {
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
       cudaGetLastError();
       return 0;
     }
-    e->kernel = kernel;
+    e.opted_in = true;
   }
-  if (e->n[cl] == 0) {
-    e->n[cl] = -1;
+  if (e.n[cl] == 0) {
+    e.n[cl] = -1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)cl);
     cfg.blockDim = dim3(kClusterThreads);
@@ -340,10 +343,10 @@ int max_active_clusters(void (*kernel)(ReduceParams), int cl) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) == cudaSuccess && n >= 1) e->n[cl] = n;
+    if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) == cudaSuccess && n >= 1) e.n[cl] = n;
     cudaGetLastError();
   }
-  return e->n[cl] > 0 ? e->n[cl] : 0;
+  return e.n[cl] > 0 ? e.n[cl] : 0;
 }
 
 // Whether the cluster kernels (CTAs of 1024 threads, one or several per row) take a matrix of M rows of N

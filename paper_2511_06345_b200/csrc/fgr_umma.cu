@@ -1,16 +1,27 @@
 // Dispatch of the tcgen05 path: picks the compiled kernel variant for a problem's activation,
 // scaling, reduction kind and Y store.  The kernel itself is in fgr_umma_kernel.cuh.
+#include <mutex>
+
 #include "fgr_umma_kernel.cuh"
 
 namespace fgr {
 
-cudaError_t umma_prepare(int) {
+// Raises the dynamic shared-memory limit of every kernel variant on the current device.  The attribute
+// belongs to (device, kernel), so the several hundred calls are made once per device ordinal; later
+// handles on that device find it done.
+cudaError_t umma_prepare(int device) {
+  constexpr int kMaxDevices = 64;
+  static std::mutex mu;
+  static bool done[kMaxDevices] = {};
+  std::lock_guard<std::mutex> lock(mu);
+  if (device >= 0 && device < kMaxDevices && done[device]) return cudaSuccess;
   cudaError_t e = umma_prepare_act_none();
   if (e == cudaSuccess) e = umma_prepare_act_relu();
   if (e == cudaSuccess) e = umma_prepare_act_gelu();
   if (e == cudaSuccess) e = umma_prepare_act_sigmoid();
   if (e == cudaSuccess) e = umma_prepare_act_tanh();
   if (e == cudaSuccess) e = umma_prepare_act_silu();
+  if (e == cudaSuccess && device >= 0 && device < kMaxDevices) done[device] = true;
   return e;
 }
 

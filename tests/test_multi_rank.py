@@ -76,6 +76,33 @@ def test_reference_arm_prints_the_contract_line():
     assert line["config"]["workload"] == "c1" and line["vs_baseline"] is None
 
 
+def test_gpus_flag_starts_the_ranks_itself():
+    """`python bench.py --gpus 2` with no launcher around it starts two ranks (torch.distributed.run on
+    127.0.0.1), they meet (gloo here: no GPU), and rank 0 alone prints a line that says n_gpus = 2."""
+    import json
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--backend", "gloo", "--plumbing-only"],
+                       env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1 and lines[0]["n_gpus"] == 2 and lines[0]["plumbing_only"] is True
+    assert lines[0]["max_over_ranks_check"] == 2.0           # ranks report 1 ms and 2 ms: the slowest one counts
+
+
+def test_both_arms_name_the_workload_with_the_same_keys():
+    """The reference arm's `config` carries the same shape keys, with the same values, as ours (built here
+    from the same helper without a GPU), for the default workload - the largest named one."""
+    import json
+    sys.path.insert(0, ROOT)
+    import bench
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1", "--warmup", "0"],
+                       capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    line = json.loads(r.stdout.strip().splitlines()[-1])
+    want = bench.shape_keys(bench.HEADLINE, bench.make_cfg(bench.HEADLINE, materialize=False))
+    assert want["workload"] == "c3" and {k: line["config"][k] for k in want} == want
+
+
 def test_bench_extra_workloads_are_well_formed():
     """The extra bench legs resolve to problems of the documented shapes (no data is generated here)."""
     sys.path.insert(0, ROOT)

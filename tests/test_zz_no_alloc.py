@@ -2,16 +2,18 @@
 whose allocator owns the GPU, a latency-critical loop, an embedding that is handed buffers only).
 It keeps its scratch in a fixed array inside the library, so it takes no workspace and no handle.
 
-Checked here through the C ABI against fgr_run on the same path, on two calls in a row: the
-second call uses other shapes and data, so anything the first call left in the shared scratch
-would show.  This file is collected last on purpose."""
+Checked here through the C ABI against fgr_run on the same path (bit for bit: same kernels, same
+tiling) and, independently, against the CPU oracle at the tolerances of the other parity tests, on
+calls in a row: each later call uses other shapes and data, so anything an earlier call left in the
+shared scratch would show.  Also checked: once the first call on the device has been made, a call
+leaves the device's free memory exactly as it found it.  This file is collected last on purpose."""
 import numpy as np
 import pytest
 import torch
 
 import fgr_inputs as gi
 import paper_2511_06345_b200 as fgr
-from parity import to_device
+from parity import compare, to_device
 
 pytestmark = pytest.mark.gpu
 
@@ -44,13 +46,18 @@ def _both(p):
 
 def _check(p):
     (y0, o0), (y1, o1) = _both(p)
-    tol = 1e-4 if p.dtype == gi.DTYPE_F32 else 2e-2          # the stated tolerances; the two paths share kernels
+    rows = p.batch * p.M
+    # against fgr_run: the same kernels in the same tiling, so not one bit may differ
     if y0 is not None:
-        assert np.abs(y1 - y0).max() <= tol * (1 + np.abs(y0).max())
-        np.testing.assert_allclose(y1, y0, rtol=tol, atol=tol)
+        assert np.array_equal(y1, y0)
     if o0 is not None:
-        np.testing.assert_allclose(o1, o0, rtol=tol, atol=tol)
-        assert not np.any(o1 == -7.0)
+        assert np.array_equal(o1, o0) and not np.any(o1 == -7.0)
+    # against the oracle, which shares nothing with either entry point: the stated tolerance and the tight bounds
+    Y = None if y1 is None else y1.astype(np.float64).reshape(rows, p.N)
+    out = None if o1 is None else o1.astype(np.float64).reshape(rows, -1)
+    worst = compare(p, Y, out, tcgen05=False)
+    official = 1e-4 if p.dtype == gi.DTYPE_F32 else 2e-2
+    assert all(v <= official for v in worst.values())
 
 
 def test_static_scratch_matches_fgr_run_twice_in_a_row(cuda_device):
@@ -63,6 +70,23 @@ def test_static_scratch_matches_fgr_run_twice_in_a_row(cuda_device):
     third = gi.make_config("c1")                              # the small named workload, max + sum-exp pairs
     third.reduce = gi.RED_MAX_SUMEXP
     _check(third)
+
+
+def test_static_scratch_leaves_free_memory_unchanged(cuda_device):
+    """After the first call on the device (which loads the module that holds the scratch array), a call
+    takes nothing from the device: free memory before == free memory after."""
+    p = gi.make_problem("m", 1, 70, 136, 40, gi.DTYPE_BF16, gi.ACT_RELU, gi.SCALE_NONE, gi.RED_MAXSUM, seed=73)
+    X, W, b, s = to_device(p)
+    out = torch.empty((p.M, 2), dtype=torch.float32, device="cuda:0")
+    desc = fgr.make_desc(p.batch, p.M, p.N, p.K, p.dtype, p.act, p.scale_kind, p.reduce)
+    fgr.fgr_run_static(desc, X, W, b, s, None, out, None)     # the warm first call
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for _ in range(3):
+        fgr.fgr_run_static(desc, X, W, b, s, None, out, None)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
 
 
 def test_static_scratch_rejects_what_does_not_fit(cuda_device):
