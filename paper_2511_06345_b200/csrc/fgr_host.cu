@@ -289,7 +289,15 @@ int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
   pi.cta_pair = cuda_cores ? 1 : p.cta_pair;
   pi.ksub = cuda_cores ? 0 : p.ksub;
   pi.launches = tf32 ? 4 : 2;   // (operand split of X and of W +) main kernel + (merge | softmax normalise)
-  pi.workspace_bytes = (uint64_t)kStatusBytes + (uint64_t)d.batch * d.M * p.parts_per_row * 8ull;
+  // tcgen05 softmax: completion counters per row-block unit (+ one finish ticket) follow the status block
+  p.head_bytes = kStatusBytes;
+  p.done_target = 0;
+  if (!cuda_cores && d.reduce == FGR_RED_SOFTMAX) {
+    const long long units = (long long)d.batch * p.tiles_m;
+    p.head_bytes += (int)align256((size_t)(units + 1) * sizeof(unsigned int));
+    p.done_target = (unsigned int)p.tiles_n * 8u * (unsigned int)p.cta_pair;   // epilogue warps per unit
+  }
+  pi.workspace_bytes = (uint64_t)p.head_bytes + (uint64_t)d.batch * d.M * p.parts_per_row * 8ull;
   if (tf32)   // the hi / lo planes of X and W follow the partial pairs, each on a 256-byte boundary
     pi.workspace_bytes = align256(align256((size_t)pi.workspace_bytes) + (size_t)d.batch * d.M * 2 * p.k_plane * 4) +
                          (uint64_t)(d.w_shared ? 1 : d.batch) * d.N * 2 * p.k_plane * 4;
@@ -416,10 +424,11 @@ int fgr_run(fgr_handle* h, const void* X, const void* W, const float* bias, cons
   p.X = X; p.W = W; p.bias = bias; p.scale_vec = scale_vec; p.Y = Y; p.out = out;
   p.R = h->residual; p.ldr = h->ldr; p.bsr = h->bsr;
   p.status = static_cast<int*>(workspace);
-  p.parts = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes);
+  p.parts = reinterpret_cast<float*>(static_cast<char*>(workspace) + p.head_bytes);
+  p.done = p.done_target ? reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) + kStatusBytes) : nullptr;
 
-  if (workspace != h->last_workspace) {   // a workspace seen for the first time: clear its status word
-    e = cudaMemsetAsync(workspace, 0, kStatusBytes, stream);
+  if (workspace != h->last_workspace) {   // a workspace seen for the first time: clear its status word (and counters)
+    e = cudaMemsetAsync(workspace, 0, (size_t)p.head_bytes, stream);
     h->last_workspace = workspace;
   }
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
@@ -436,7 +445,7 @@ int fgr_run(fgr_handle* h, const void* X, const void* W, const float* bias, cons
   if (tf32 && e == cudaSuccess) {
     // split X and W into tf32 hi / lo planes inside the workspace (ahead of the timed main kernel)
     char* wsb = static_cast<char*>(workspace);
-    const size_t x_off = align256((size_t)kStatusBytes + (size_t)d.batch * d.M * p.parts_per_row * 8u);
+    const size_t x_off = align256((size_t)p.head_bytes + (size_t)d.batch * d.M * p.parts_per_row * 8u);
     const size_t w_off = align256(x_off + (size_t)d.batch * d.M * 2 * p.k_plane * 4);
     xp = reinterpret_cast<float*>(wsb + x_off);
     wp = reinterpret_cast<float*>(wsb + w_off);
@@ -522,7 +531,8 @@ int fgr_get_status(fgr_handle* h) {
     rc = FGR_ERR_CUDA;
   } else if (word != 0) {
     rc = word;
-    cudaMemset(h->last_workspace, 0, sizeof word);   // reported once
+    // reported once; a run that gave up may also have left its completion counters half counted
+    cudaMemset(h->last_workspace, 0, (size_t)h->base.head_bytes);
   }
   if (prev != h->desc.device && prev >= 0) cudaSetDevice(prev);
   return rc;

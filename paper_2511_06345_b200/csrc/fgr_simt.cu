@@ -270,13 +270,7 @@ __global__ void __launch_bounds__(256) merge_kernel(const Params p) {
 // leaves the factor exp(m_slot - m_row) / l_row of every slot in shared memory; then the CTA
 // rescales the row with 16-byte accesses.
 template <typename T>
-__global__ void __launch_bounds__(256) normalise_kernel(const Params p) {
-  extern __shared__ float factor[];   // [parts_per_row]
-  let_next_kernel_start();
-  wait_for_prior_kernel();
-  // The GEMM pass writes rows in ascending order, so the rows written last are the ones still in L2:
-  // take them first, before this pass's own traffic evicts them.
-  const long long row = (long long)gridDim.x - 1 - blockIdx.x;
+__device__ __forceinline__ void normalise_row(const Params& p, long long row, float* factor) {
   const int bt = (int)(row / p.M), m = (int)(row % p.M);
   const float2* src = reinterpret_cast<const float2*>(p.parts) + row * p.parts_per_row;
   if (threadIdx.x < 32) {
@@ -359,6 +353,178 @@ __global__ void __launch_bounds__(256) normalise_kernel(const Params p) {
   }
 }
 
+// Softmax, second pass after the CUDA-core main kernel: waits for that kernel to end, then one CTA per row,
+// last rows first (the main kernel writes rows in ascending order, so the rows written last are the ones
+// still in L2).
+template <typename T>
+__global__ void __launch_bounds__(256) normalise_kernel(const Params p) {
+  extern __shared__ float factor[];   // [parts_per_row]
+  let_next_kernel_start();
+  wait_for_prior_kernel();
+  normalise_row<T>(p, (long long)gridDim.x - 1 - blockIdx.x, factor);
+}
+
+// Softmax, second pass beside the tcgen05 main kernel.  This kernel is launched as the main kernel's
+// programmatic dependent and does not wait for it to end: its CTAs start once every CTA of the main kernel
+// has started (or ended), find room next to them on the SMs (40 registers a thread, 16 bytes of shared
+// memory: two CTAs fit beside a main-kernel CTA), and rescale each block of rows as soon as the main kernel
+// has published it (p.done), while the stored exponentials are still in L2.  The second pass then costs no
+// DRAM read and hides behind the main kernel, except for the rows of the main kernel's last tiles.  The
+// main kernel never waits for this one, so the wait below always ends; it is bounded all the same (about a
+// second, or as soon as the status word shows that something gave up), after which the CTA leaves its row
+// untouched.
+//
+// A CTA per row, rows in ascending order (the order in which the main kernel finishes them).  Thread 0 polls
+// the row block's counter with acquire loads.  Then every thread issues the loads of its part of the row
+// BEFORE the row's statistics exist (they do not depend on them), warp 0 merges the row's partial pairs
+// (lanes stride over them, fixed shuffle tree: bit-identical from run to run) and broadcasts (m_row, 1 / l_row),
+// and each thread rescales what it loaded by exp(m_slot - m_row) / l_row, the slot's pair coming from L1.
+// The next kernel in the stream is let in only when a CTA is done: until then the rows of the main kernel's
+// last tiles have the SMs to themselves (that tail is the one part of this pass that nothing hides).
+// The last CTA to finish zeroes the counters for the next run.
+constexpr long long kChaseWaitCycles = 2000000000LL;   // about one second at ~2 GHz
+constexpr int kChaseThreads = 256;
+
+__device__ __forceinline__ unsigned int load_acquire(const unsigned int* p) {
+  unsigned int v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint32_t scale_bf16x2(uint32_t w, float f) {
+  __nv_bfloat162 r = __floats2bfloat162_rn(__uint_as_float(w << 16) * f, __uint_as_float(w & 0xffff0000u) * f);
+  return *reinterpret_cast<uint32_t*>(&r);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kChaseThreads) normalise_chase_kernel(const Params p) {
+  __shared__ int flag;
+  __shared__ float stat[2];   // (m_row, 1 / l_row)
+  const int lane = threadIdx.x & 31;
+  const long long row = blockIdx.x;
+  if (threadIdx.x == 0) {
+    const long long unit = (row / p.M) * p.tiles_m + (row % p.M) / (kUmmaTileM * p.cta_pair);
+    int ok = 1;
+    if (load_acquire(p.done + unit) < p.done_target) {
+      const long long t0 = clock64();
+      for (unsigned int ns = 128;; ns = ns < 1024 ? 2 * ns : ns) {
+        __nanosleep(ns);
+        if (load_acquire(p.done + unit) >= p.done_target) break;
+        if (*reinterpret_cast<volatile int*>(p.status) != 0) { ok = 0; break; }   // the main kernel (or another CTA) gave up
+        if (clock64() - t0 > kChaseWaitCycles) { atomicExch(p.status, (int)FGR_ERR_DEVICE_TIMEOUT); ok = 0; break; }
+      }
+    }
+    flag = ok;
+  }
+  __syncthreads();
+  if (flag) {
+    const float2* src = reinterpret_cast<const float2*>(p.parts) + row * p.parts_per_row;
+    const int bt = (int)(row / p.M), m = (int)(row % p.M);
+    T* y = static_cast<T*>(p.Y) + (long long)bt * p.bsy + (long long)m * p.ldy;
+    auto stats = [&]() {   // warp 0: (m_row, l_row) from the partial pairs
+      float a = -CUDART_INF_F;
+      for (int t = lane; t < p.parts_per_row; t += 32) a = fmaxf(a, src[t].x);
+#pragma unroll
+      for (int o = 16; o >= 1; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+      float l = 0.0f;
+      for (int t = lane; t < p.parts_per_row; t += 32) {
+        const float2 v = src[t];
+        if (v.x > -CUDART_INF_F) l += v.y * expf(v.x - a);
+      }
+#pragma unroll
+      for (int o = 16; o >= 1; o >>= 1) {
+        const float ol = __shfl_xor_sync(0xffffffffu, l, o);
+        l = (lane & o) ? ol + l : l + ol;
+      }
+      if (lane == 0) {
+        stat[0] = a;
+        stat[1] = 1.0f / l;
+        // optional row statistics (row max, sum of exp(y - max)): what a combine over column shards needs
+        if (p.out) reinterpret_cast<float2*>(p.out)[row] = make_float2(a, l);
+      }
+    };
+    auto factor_at = [&](int c) {
+      const float ms = src[part_slot(c, p.tile_n, p.half_n, p.slots_per_tile)].x;
+      return ms > -CUDART_INF_F ? expf(ms - stat[0]) * stat[1] : 0.0f;
+    };
+    constexpr int U = 2;                       // accesses in flight per thread
+    bool wide = false;
+    if constexpr (sizeof(T) == 2) wide = (reinterpret_cast<uintptr_t>(y) & 31u) == 0 && p.N % 16 == 0;
+    bool have_stats = false;
+    if (wide) {
+      // bf16 rows that start on a 32-byte boundary: 256-bit accesses (16 elements, inside one slot)
+      for (int c0 = threadIdx.x * 16; c0 < p.N || !have_stats; c0 += U * kChaseThreads * 16) {
+        uint32_t w[U][8];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const int c = c0 + u * kChaseThreads * 16;
+          if (c < p.N)
+            asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                         : "=r"(w[u][0]), "=r"(w[u][1]), "=r"(w[u][2]), "=r"(w[u][3]), "=r"(w[u][4]), "=r"(w[u][5]), "=r"(w[u][6]),
+                           "=r"(w[u][7])
+                         : "l"(y + c)
+                         : "memory");
+        }
+        if (!have_stats) {                     // uniform across the CTA: the first trip of every thread
+          if (threadIdx.x < 32) stats();
+          __syncthreads();
+          have_stats = true;
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const int c = c0 + u * kChaseThreads * 16;
+          if (c < p.N) {
+            const float f = factor_at(c);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) w[u][j] = scale_bf16x2(w[u][j], f);
+            asm volatile("st.global.cs.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(y + c), "r"(w[u][0]), "r"(w[u][1]),
+                         "r"(w[u][2]), "r"(w[u][3]), "r"(w[u][4]), "r"(w[u][5]), "r"(w[u][6]), "r"(w[u][7])
+                         : "memory");
+          }
+        }
+      }
+    } else {
+      constexpr int V = 16 / (int)sizeof(T);   // elements per 16-byte access; N is a multiple of V, slot edges of 16
+      for (int c0 = threadIdx.x * V; c0 < p.N || !have_stats; c0 += U * kChaseThreads * V) {
+        uint4 w[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const int c = c0 + u * kChaseThreads * V;
+          if (c < p.N) w[u] = *reinterpret_cast<const uint4*>(y + c);
+        }
+        if (!have_stats) {
+          if (threadIdx.x < 32) stats();
+          __syncthreads();
+          have_stats = true;
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const int c = c0 + u * kChaseThreads * V;
+          if (c < p.N) {
+            const float f = factor_at(c);
+            if constexpr (sizeof(T) == 4) {
+              float* v = reinterpret_cast<float*>(&w[u]);
+#pragma unroll
+              for (int j = 0; j < 4; ++j) v[j] *= f;
+            } else {
+              w[u].x = scale_bf16x2(w[u].x, f); w[u].y = scale_bf16x2(w[u].y, f);
+              w[u].z = scale_bf16x2(w[u].z, f); w[u].w = scale_bf16x2(w[u].w, f);
+            }
+            *reinterpret_cast<uint4*>(y + c) = w[u];
+          }
+        }
+      }
+    }
+  }
+  __syncthreads();
+  let_next_kernel_start();
+  // finish ticket: whoever draws the last one knows that no CTA will read a counter again
+  const long long units = (long long)p.batch * p.tiles_m;
+  if (threadIdx.x == 0) flag = atomicAdd(p.done + units, 1u) == gridDim.x - 1 ? 1 : 0;
+  __syncthreads();
+  if (flag)
+    for (long long u = threadIdx.x; u <= units; u += blockDim.x) p.done[u] = 0u;
+}
+
 }  // namespace
 
 cudaError_t launch_simt(const Params& p, cudaStream_t stream) {
@@ -396,6 +562,10 @@ cudaError_t launch_merge(const Params& p, cudaStream_t stream) {
 
 cudaError_t launch_normalise(const Params& p, cudaStream_t stream) {
   const long long rows = (long long)p.batch * p.M;
+  if (p.done) {   // beside the tcgen05 main kernel
+    if (p.dtype == FGR_F32) return launch_dependent(normalise_chase_kernel<float>, (unsigned)rows, kChaseThreads, 0, stream, p);
+    return launch_dependent(normalise_chase_kernel<__nv_bfloat16>, (unsigned)rows, kChaseThreads, 0, stream, p);
+  }
   const size_t smem = (size_t)p.parts_per_row * sizeof(float);
   if (p.dtype == FGR_F32) return launch_dependent(normalise_kernel<float>, (unsigned)rows, 256, smem, stream, p);
   return launch_dependent(normalise_kernel<__nv_bfloat16>, (unsigned)rows, 256, smem, stream, p);

@@ -550,8 +550,24 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
     const int c_end = half ? p.tile_n : p.half_n;
     uint32_t tcount = 0;
     bool ok = true;
+    // Softmax: the normalise kernel runs beside this one and rescales a block of rows once every tile of
+    // it is stored.  A warp publishes a finished tile one tile late: by then the tile's stores have long
+    // been acknowledged, so the fence below finds nothing to wait for (a fence right after the stores
+    // stalls the warp until the last of them has drained).
+    long long unpublished = -1;             // row-block unit of the tile this warp has stored but not yet published
+    auto publish = [&]() {
+      if constexpr (V::kSoftmax) {
+        if (unpublished >= 0) {
+          __threadfence();                  // every lane: its stores of that tile before the count below
+          __syncwarp();
+          if (lane == 0) atomicAdd(p.done + unpublished, 1u);
+          unpublished = -1;
+        }
+      }
+    };
     for (long long t = unit0; t < p.num_tiles && ok; t += unit_step, ++tcount) {
       const TileCoord c = tile_coord(t, p, rank);
+      publish();
       // stage the bias and scale of this warp's columns in its own slice of shared memory
       for (int i = lane; i < c_end - c_begin; i += 32) {
         const int n = c.n0 + c_begin + i;
@@ -738,7 +754,11 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
         float2* dst = reinterpret_cast<float2*>(p.parts) + ((long long)c.bt * p.M + m) * p.parts_per_row + tn * 2 + half;
         *dst = make_float2(r0, r1);
       }
+      if constexpr (V::kSoftmax) {
+        if (p.done) unpublished = t / p.tiles_n;
+      }
     }
+    if (ok) publish();
   }
 
   tcgen05_fence_before();
