@@ -45,10 +45,10 @@ struct Params {
   int w_shared;        // 1: W is one [N, K] matrix used by every batch element (bsw = 0)
   int chunk_blocks;    // 3xTF32 path: 32-wide k-blocks accumulated in tensor memory before the epilogue adds them up
   // Softmax on the tcgen05 paths: the normalise kernel runs beside the main kernel and rescales a block of rows
-  // as soon as all its tiles are stored.  done[u] counts the epilogue warps that have finished (and published)
-  // a tile of row-block unit u = tile index / tiles_n; a unit is complete at done_target.  done[num_units] is
-  // the finish ticket of the normalise kernel, whose last CTA zeroes the array for the next run.  Null
-  // elsewhere: the second kernel then simply waits for the first to end.
+  // as soon as all its tiles are stored.  done[u] (in the workspace head) counts the epilogue warps that have
+  // finished and published a tile of row-block unit u = tile index / tiles_n; a unit is complete at
+  // done_target.  done[num_units] is the finish ticket of the normalise kernel, whose last CTA zeroes the array
+  // for the next run.  Null elsewhere: the second kernel then simply waits for the first to end.
   unsigned int* done;
   unsigned int done_target;
   int head_bytes;      // workspace bytes ahead of the partial pairs: status block (+ the counters above)

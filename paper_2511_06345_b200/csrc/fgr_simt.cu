@@ -189,11 +189,9 @@ __device__ __forceinline__ void let_next_kernel_start() { asm volatile("griddepc
 // order, then a fixed xor-shuffle tree combines the G lanes.  The order never depends on timing:
 // bit-identical results from run to run.
 template <int G>
-__global__ void __launch_bounds__(256) merge_kernel(const Params p) {
-  let_next_kernel_start();
-  wait_for_prior_kernel();
+__device__ __forceinline__ void merge_rows(const Params& p, long long block) {
   const int lane = threadIdx.x & 31, sub = lane % G;
-  const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const long long warp = block * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const long long row = warp * (32 / G) + lane / G;
   const bool row_ok = row < (long long)p.batch * p.M;
   const float2* src = reinterpret_cast<const float2*>(p.parts) + (row_ok ? row : 0) * p.parts_per_row;
@@ -232,6 +230,7 @@ __global__ void __launch_bounds__(256) merge_kernel(const Params p) {
   }
   const bool exp_kind = p.reduce != FGR_RED_MAXSUM;
   float a = -CUDART_INF_F, b = 0.0f;
+#pragma unroll 4
   for (int t = sub; t < p.parts_per_row; t += G) {
     float2 v = src[t];
     if (exp_kind) {
@@ -263,6 +262,13 @@ __global__ void __launch_bounds__(256) merge_kernel(const Params p) {
     if (p.reduce == FGR_RED_LSE) p.out[row] = a + logf(b);
     else if (p.reduce != FGR_RED_SOFTMAX) reinterpret_cast<float2*>(p.out)[row] = make_float2(a, b);
   }
+}
+
+template <int G>
+__global__ void __launch_bounds__(256) merge_kernel(const Params p) {
+  let_next_kernel_start();
+  wait_for_prior_kernel();
+  merge_rows<G>(p, blockIdx.x);
 }
 
 // Softmax, second pass.  The GEMM pass stored E[m, n] = exp(y - m_slot) per partial slot together
@@ -554,9 +560,12 @@ cudaError_t launch_dependent(Kernel kernel, unsigned grid, unsigned block, size_
 
 cudaError_t launch_merge(const Params& p, cudaStream_t stream) {
   const long long rows = (long long)p.batch * p.M;
-  // lanes per row: enough to cover the partial pairs of a row, so that few lanes idle
-  if (p.parts_per_row <= 2) return launch_dependent(merge_kernel<2>, (unsigned)((rows + 127) / 128), 256, 0, stream, p);
-  if (p.parts_per_row <= 16) return launch_dependent(merge_kernel<8>, (unsigned)((rows + 31) / 32), 256, 0, stream, p);
+  // Lanes per row: few, each folding up to eight pairs (its loads are independent and go out together), so that
+  // the grid stays small.  The next run's main kernel, a programmatic dependent of this one, may move in only
+  // once every CTA here has started; a grid that fits beside the main kernel in one wave (two CTAs per SM) lets
+  // it do so while the main kernel's CTAs are still leaving.
+  if (p.parts_per_row <= 8) return launch_dependent(merge_kernel<2>, (unsigned)((rows + 127) / 128), 256, 0, stream, p);
+  if (p.parts_per_row <= 64) return launch_dependent(merge_kernel<8>, (unsigned)((rows + 31) / 32), 256, 0, stream, p);
   return launch_dependent(merge_kernel<32>, (unsigned)((rows + 7) / 8), 256, 0, stream, p);
 }
 

@@ -190,6 +190,9 @@ __device__ __forceinline__ void tcgen05_mma_tf32_pair(uint32_t d_tmem, uint64_t 
       : "memory");
 }
 
+// Release / acquire fence at device scope (lighter than __threadfence(), the sequentially consistent one).
+__device__ __forceinline__ void fence_acq_rel_gpu() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
+
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
@@ -550,15 +553,15 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
     const int c_end = half ? p.tile_n : p.half_n;
     uint32_t tcount = 0;
     bool ok = true;
-    // Softmax: the normalise kernel runs beside this one and rescales a block of rows once every tile of
-    // it is stored.  A warp publishes a finished tile one tile late: by then the tile's stores have long
-    // been acknowledged, so the fence below finds nothing to wait for (a fence right after the stores
-    // stalls the warp until the last of them has drained).
+    // Softmax: the normalise kernel runs beside this one and rescales a block of rows once every tile of it is
+    // stored; a warp adds 1 to the count of its tile's row block.  It does so after it has waited for the
+    // accumulator of its next tile (or has none left): the fence that must precede the count then finds the
+    // tile's stores acknowledged, where a fence right after them stalls the warp until the last has drained.
     long long unpublished = -1;             // row-block unit of the tile this warp has stored but not yet published
     auto publish = [&]() {
       if constexpr (V::kSoftmax) {
         if (unpublished >= 0) {
-          __threadfence();                  // every lane: its stores of that tile before the count below
+          fence_acq_rel_gpu();              // every lane: its stores of that tile before the count below
           __syncwarp();
           if (lane == 0) atomicAdd(p.done + unpublished, 1u);
           unpublished = -1;
@@ -567,7 +570,6 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
     };
     for (long long t = unit0; t < p.num_tiles && ok; t += unit_step, ++tcount) {
       const TileCoord c = tile_coord(t, p, rank);
-      publish();
       // stage the bias and scale of this warp's columns in its own slice of shared memory
       for (int i = lane; i < c_end - c_begin; i += 32) {
         const int n = c.n0 + c_begin + i;
@@ -626,6 +628,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
       const uint32_t buf = tcount & 1u, aph = (tcount >> 1) & 1u;
       ok = __all_sync(0xffffffffu, mbar_wait(tmem_full_bar(buf), aph, abort_flag, p.status));
       if (!ok) break;
+      publish();   // the previous tile: its stores went out before the wait above, nothing new has been stored since
       tcgen05_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * 256u;
       using OutT = typename std::conditional<TF32, float, __nv_bfloat16>::type;
@@ -755,7 +758,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
         *dst = make_float2(r0, r1);
       }
       if constexpr (V::kSoftmax) {
-        if (p.done) unpublished = t / p.tiles_n;
+        if (p.done) unpublished = t / p.tiles_n;                     // row block (of 128 rows, or 256 for a CTA pair)
       }
     }
     if (ok) publish();
