@@ -14,6 +14,7 @@
 using namespace fgr;
 
 namespace {
+constexpr int kHostChunks = 4;
 constexpr int kMapSlots = 8;
 struct MapCache {
   const void* key[kMapSlots];
@@ -57,6 +58,16 @@ struct fgr_handle {
   void* stage[7];
   size_t stage_bytes[7];
   cudaStream_t host_stream;
+  // fgr_run_host in chunks: sub-handles for blocks of rows (or of batches), their workspaces (slices of one
+  // allocation), a stream for each copy direction and the events that chain copy -> run -> copy
+  fgr_handle* sub[kHostChunks];
+  long long sub_first[kHostChunks + 1];   // first row (batch == 1) or first batch of each chunk
+  int sub_count;                          // 0 = not planned yet, 1 = whole problem in one piece
+  bool sub_by_batch;
+  void* sub_ws;
+  size_t sub_ws_bytes, sub_ws_off[kHostChunks];
+  cudaStream_t in_stream, out_stream;
+  cudaEvent_t ev_in[kHostChunks], ev_run[kHostChunks], ev_shared;
   // optional timing of the main kernel
   bool profiling;
   std::vector<cudaEvent_t>* events;   // pairs (before, after)
@@ -538,6 +549,57 @@ int fgr_get_status(fgr_handle* h) {
   return rc;
 }
 
+// Plans fgr_run_host's chunks once per handle: kHostChunks blocks of batches when there are at least that
+// many, else (one batch, plain GEMM, enough rows) blocks of rows in multiples of 256.  Each chunk gets a
+// sub-handle of its own shape with the parent's strides spelled out, so it runs on a slice of the parent's
+// staging buffers.  Returns false if the problem stays in one piece.
+static bool plan_host_chunks(fgr_handle* h) {
+  if (h->sub_count) return h->sub_count > 1;
+  h->sub_count = 1;
+  const fgr_desc& d = h->desc;
+  const Params& b = h->base;
+  if (d.conv_taps > 1) return false;   // overlapping rows: the chunks' input copies would overlap too
+  long long total, unit;
+  if (d.batch >= kHostChunks) { h->sub_by_batch = true; total = d.batch; unit = 1; }
+  else if (d.batch == 1 && d.M >= kHostChunks * 256) { h->sub_by_batch = false; total = d.M; unit = 256; }
+  else return false;
+  const long long per = ((total + kHostChunks - 1) / kHostChunks + unit - 1) / unit * unit;
+  // a chunk's slice of `out` must start on an 8-byte boundary
+  if ((per * (h->sub_by_batch ? d.M : 1) * out_width(d.reduce)) % 2 != 0) return false;
+  int n = 0;
+  for (long long first = 0; first < total && n < kHostChunks; first += per) h->sub_first[n++] = first;
+  h->sub_first[n] = total;
+  size_t ws = 0;
+  for (int c = 0; c < n; ++c) {
+    fgr_desc sd = d;
+    const int count = (int)(h->sub_first[c + 1] - h->sub_first[c]);
+    if (h->sub_by_batch) sd.batch = count; else sd.M = count;
+    sd.ldx = b.ldx; sd.ldw = b.ldw; sd.ldy = b.ldy;
+    sd.bsx = b.bsx; sd.bsw = b.bsw; sd.bsy = b.bsy;
+    if (fgr_create(&sd, &h->sub[c]) != FGR_OK) {
+      for (int k = 0; k < c; ++k) { fgr_destroy(h->sub[k]); h->sub[k] = nullptr; }
+      return false;
+    }
+    h->sub_ws_off[c] = ws;
+    ws += align256((size_t)h->sub[c]->plan.workspace_bytes);
+  }
+  bool ok = cudaMalloc(&h->sub_ws, ws) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&h->in_stream, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&h->out_stream, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&h->ev_shared, cudaEventDisableTiming) == cudaSuccess;
+  for (int c = 0; c < n && ok; ++c)
+    ok = cudaEventCreateWithFlags(&h->ev_in[c], cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&h->ev_run[c], cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) {   // leave what exists to fgr_destroy; run in one piece
+    cudaGetLastError();
+    for (int c = 0; c < n; ++c) { fgr_destroy(h->sub[c]); h->sub[c] = nullptr; }
+    return false;
+  }
+  h->sub_ws_bytes = ws;
+  h->sub_count = n;
+  return n > 1;
+}
+
 int fgr_run_host(fgr_handle* h, const void* X, const void* W, const float* bias, const float* scale_vec, void* Y,
                  float* out) {
   if (!h || !X || !W) return FGR_ERR_INVALID_ARG;
@@ -573,6 +635,57 @@ int fgr_run_host(fgr_handle* h, const void* X, const void* W, const float* bias,
       if (i == 0) h->maps_x.clear();   // (the maps are keyed by address; a handle's strides never change, so a
       if (i == 1) h->maps_w.clear();   //  reused address would still be described correctly: this is tidiness)
     }
+  }
+  if (rc == FGR_OK && plan_host_chunks(h)) {
+    // Chunked: the copy in of chunk c + 1, the kernels of chunk c and the copy out of chunk c - 1 overlap
+    // (three streams, events in between).  What all chunks share (bias, scale; W unless it is batched) goes first.
+    const size_t ex = e;
+    const int n = h->sub_count;
+    auto fail = [&](cudaError_t ce) { if (ce != cudaSuccess && rc == FGR_OK) rc = FGR_ERR_CUDA; };
+    if (want[2]) fail(cudaMemcpyAsync(h->stage[2], bias, want[2], cudaMemcpyHostToDevice, h->in_stream));
+    if (want[3]) fail(cudaMemcpyAsync(h->stage[3], scale_vec, want[3], cudaMemcpyHostToDevice, h->in_stream));
+    const bool w_chunked = h->sub_by_batch && !d.w_shared;
+    if (!w_chunked) fail(cudaMemcpyAsync(h->stage[1], W, want[1], cudaMemcpyHostToDevice, h->in_stream));
+    fail(cudaEventRecord(h->ev_shared, h->in_stream));
+    fail(cudaStreamWaitEvent(h->host_stream, h->ev_shared, 0));
+    for (int c = 0; c < n && rc == FGR_OK; ++c) {
+      const long long first = h->sub_first[c], count = h->sub_first[c + 1] - first;
+      const size_t x_off = (size_t)first * (h->sub_by_batch ? b.bsx : b.ldx) * ex;
+      const size_t y_off = (size_t)first * (h->sub_by_batch ? b.bsy : b.ldy) * ex;
+      const size_t w_off = w_chunked ? (size_t)first * b.bsw * ex : 0;
+      const size_t rows_before = (size_t)first * (h->sub_by_batch ? d.M : 1);
+      const size_t rows_here = (size_t)count * (h->sub_by_batch ? d.M : 1);
+      // bytes of this chunk's slices (the last row of a slice ends at its K or N, not at the next stride)
+      const size_t x_bytes = h->sub_by_batch ? ((size_t)(count - 1) * b.bsx + (size_t)(d.M - 1) * b.ldx + d.K) * ex
+                                             : ((size_t)(count - 1) * b.ldx + d.K) * ex;
+      const size_t w_bytes = ((size_t)(count - 1) * b.bsw + (size_t)(d.N - 1) * b.ldw + d.K) * ex;
+      const size_t y_bytes = h->sub_by_batch ? ((size_t)(count - 1) * b.bsy + (size_t)(d.M - 1) * b.ldy + d.N) * ex
+                                             : ((size_t)(count - 1) * b.ldy + d.N) * ex;
+      char* dx = static_cast<char*>(h->stage[0]) + x_off;
+      char* dw = static_cast<char*>(h->stage[1]) + w_off;
+      char* dy = need_y ? static_cast<char*>(h->stage[4]) + y_off : nullptr;
+      float* dout = softmax ? nullptr : static_cast<float*>(h->stage[5]) + rows_before * out_width(d.reduce);
+      const float* dbias = bias ? static_cast<const float*>(h->stage[2]) + (d.bias_per_batch && h->sub_by_batch ? (size_t)first * d.N : 0) : nullptr;
+      fail(cudaMemcpyAsync(dx, static_cast<const char*>(X) + x_off, x_bytes, cudaMemcpyHostToDevice, h->in_stream));
+      if (w_chunked) fail(cudaMemcpyAsync(dw, static_cast<const char*>(W) + w_off, w_bytes, cudaMemcpyHostToDevice, h->in_stream));
+      fail(cudaEventRecord(h->ev_in[c], h->in_stream));
+      fail(cudaStreamWaitEvent(h->host_stream, h->ev_in[c], 0));
+      if (rc == FGR_OK)
+        rc = fgr_run(h->sub[c], dx, dw, dbias, scale_vec ? static_cast<float*>(h->stage[3]) : nullptr, dy, dout,
+                     static_cast<char*>(h->sub_ws) + h->sub_ws_off[c], (size_t)h->sub[c]->plan.workspace_bytes, h->host_stream);
+      fail(cudaEventRecord(h->ev_run[c], h->host_stream));
+      fail(cudaStreamWaitEvent(h->out_stream, h->ev_run[c], 0));
+      if (need_y) fail(cudaMemcpyAsync(static_cast<char*>(Y) + y_off, dy, y_bytes, cudaMemcpyDeviceToHost, h->out_stream));
+      if (!softmax)
+        fail(cudaMemcpyAsync(out + rows_before * out_width(d.reduce), dout, rows_here * out_width(d.reduce) * 4, cudaMemcpyDeviceToHost, h->out_stream));
+    }
+    if (cudaStreamSynchronize(h->out_stream) != cudaSuccess || cudaStreamSynchronize(h->in_stream) != cudaSuccess) { cudaGetLastError(); rc = FGR_ERR_CUDA; }
+    for (int c = 0; c < n; ++c) {
+      const int st = fgr_get_status(h->sub[c]);
+      if (rc == FGR_OK && st != FGR_OK) rc = st;
+    }
+    if (prev != d.device && prev >= 0) cudaSetDevice(prev);
+    return rc;
   }
   cudaStream_t s = h->host_stream;
   const void* src[4] = {X, W, bias, scale_vec};
@@ -635,7 +748,8 @@ int fgr_profile_empty_launches(int n, int device, void* cuda_stream) {
 
 int fgr_destroy(fgr_handle* h) {
   if (!h) return FGR_OK;
-  bool owns = h->host_stream != nullptr || !h->events->empty();
+  for (int c = 0; c < kHostChunks; ++c) if (h->sub[c]) fgr_destroy(h->sub[c]);
+  bool owns = h->host_stream != nullptr || !h->events->empty() || h->sub_ws || h->in_stream || h->out_stream || h->ev_shared;
   for (int i = 0; i < 7; ++i) owns = owns || h->stage[i];
   if (owns) {
     int prev = -1;
@@ -643,6 +757,14 @@ int fgr_destroy(fgr_handle* h) {
     if (prev != h->desc.device) cudaSetDevice(h->desc.device);
     if (h->host_stream) { cudaStreamSynchronize(h->host_stream); cudaStreamDestroy(h->host_stream); }
     for (int i = 0; i < 7; ++i) if (h->stage[i]) cudaFree(h->stage[i]);
+    if (h->in_stream) { cudaStreamSynchronize(h->in_stream); cudaStreamDestroy(h->in_stream); }
+    if (h->out_stream) { cudaStreamSynchronize(h->out_stream); cudaStreamDestroy(h->out_stream); }
+    if (h->sub_ws) cudaFree(h->sub_ws);
+    if (h->ev_shared) cudaEventDestroy(h->ev_shared);
+    for (int c = 0; c < kHostChunks; ++c) {
+      if (h->ev_in[c]) cudaEventDestroy(h->ev_in[c]);
+      if (h->ev_run[c]) cudaEventDestroy(h->ev_run[c]);
+    }
     for (cudaEvent_t ev : *h->events) cudaEventDestroy(ev);
     if (prev != h->desc.device && prev >= 0) cudaSetDevice(prev);
   }

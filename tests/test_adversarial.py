@@ -126,6 +126,36 @@ def test_host_buffer_entry_point(cuda_device):
         fgr.fgr_destroy(h)
 
 
+def test_host_buffer_entry_point_in_chunks(cuda_device):
+    """fgr_run_host splits large problems into four chunks (blocks of rows, or of batches) whose copies and
+    kernels overlap on three streams; the chunks must tile the problem exactly.  Shapes: ragged row blocks
+    (1100 rows -> 512 + 512 + 76), batches that do not divide by four (6 -> 2 + 2 + 2), per-batch bias,
+    softmax (P and no `out`), LSE (one float per row: the chunks' slices of `out` stay 8-byte aligned)."""
+    cases = [
+        gi.make_config("c2", M=1100, N=520, K=136),
+        gi.make_config("c3", M=1030, N=264, K=72, scale=3.0),
+        gi.make_config("c5", batch=6, M=130, N=264, K=72, bias_per_batch=1),
+        gi.make_config("c4", batch=5, M=64, N=520, K=136, write_y=1),
+        gi.make_config("c1", M=1024, N=136, K=64, write_y=1),
+    ]
+    for p in cases:
+        desc = fgr.make_desc(p.batch, p.M, p.N, p.K, p.dtype, p.act, p.scale_kind, p.reduce, scale=p.scale,
+                             write_y=p.write_y, bias_per_batch=p.bias_per_batch)
+        h = fgr.fgr_create(desc)
+        rows = p.batch * p.M
+        need_y = bool(p.write_y) or p.reduce == gi.RED_SOFTMAX
+        ydt = np.float32 if p.dtype == gi.DTYPE_F32 else np.uint16
+        for _ in range(2):
+            Y = np.zeros((rows, p.N), ydt) if need_y else None
+            out = np.full((rows, max(p.out_width, 1)), -7.0, np.float32) if p.out_width else None
+            ptr = lambda a: None if a is None else a.ctypes.data
+            assert fgr.fgr_run_host(h, ptr(p.X), ptr(p.W), ptr(p.bias), ptr(p.scale_vec), ptr(Y), ptr(out)) == fgr.FGR_OK
+            Yf = None if Y is None else (Y if p.dtype == gi.DTYPE_F32 else gi.bf16_bits_to_f32(Y).reshape(Y.shape)).astype(np.float64)
+            compare(p, Yf, None if out is None else out.astype(np.float64), tcgen05=p.dtype == gi.DTYPE_BF16)
+            assert out is None or not np.any(out == -7.0)
+        fgr.fgr_destroy(h)
+
+
 def test_null_and_misaligned_pointers_are_rejected(cuda_device):
     p = gi.make_config("c2", M=130, N=264, K=72)
     X, W, b, s = to_device(p)
