@@ -307,6 +307,12 @@ int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
     const long long units = (long long)d.batch * p.tiles_m;
     p.head_bytes += (int)align256((size_t)(units + 1) * sizeof(unsigned int));
     p.done_target = (unsigned int)p.tiles_n * 8u * (unsigned int)p.cta_pair;   // epilogue warps per unit
+  } else if (path == FGR_PATH_SIMT && d.reduce != FGR_RED_SOFTMAX) {
+    // CUDA-core tiles: one counter per block of 64 rows; the CTA that completes a block merges its rows, so
+    // there is no second launch (these are the small problems, bound by launch latency)
+    p.head_bytes += (int)align256((size_t)d.batch * p.tiles_m * sizeof(unsigned int));
+    p.done_target = (unsigned int)p.tiles_n;
+    pi.launches = 1;
   }
   pi.workspace_bytes = (uint64_t)p.head_bytes + (uint64_t)d.batch * d.M * p.parts_per_row * 8ull;
   if (tf32)   // the hi / lo planes of X and W follow the partial pairs, each on a 256-byte boundary
@@ -507,7 +513,10 @@ int fgr_run(fgr_handle* h, const void* X, const void* W, const float* bias, cons
     e = cudaEventRecord(ev1, stream);
     h->events_used += 2;
   }
-  if (rc == FGR_OK && e == cudaSuccess) e = softmax ? launch_normalise(p, stream) : launch_merge(p, stream);
+  if (rc == FGR_OK && e == cudaSuccess) {
+    if (softmax) e = launch_normalise(p, stream);
+    else if (h->plan.path != FGR_PATH_SIMT) e = launch_merge(p, stream);   // (the CUDA-core GEMM kernel merges its own pairs)
+  }
   if (e != cudaSuccess) { cudaGetLastError(); rc = FGR_ERR_CUDA; }
   h->last_stream = stream;
   h->ran = true;

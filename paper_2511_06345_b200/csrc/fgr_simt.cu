@@ -12,7 +12,7 @@
 namespace fgr {
 namespace {
 
-constexpr int BK = 16;
+constexpr int BK = 32;
 constexpr int PAD = 4;
 
 __device__ __forceinline__ float4 load4(const float* p) { return *reinterpret_cast<const float4*>(p); }
@@ -61,6 +61,95 @@ __device__ __forceinline__ float group16_sum(float v) {
   return v;
 }
 
+// Programmatic dependent launch: the kernels below may be made resident while the kernel before
+// them in the stream is still running; this wait returns once that kernel has completed and its
+// writes are visible.  (A no-op for a kernel launched the ordinary way.)
+__device__ __forceinline__ void wait_for_prior_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel in the stream (if it was launched as a programmatic dependent) become
+// resident now and run its set-up; it still waits for this grid to finish before touching memory.
+__device__ __forceinline__ void let_next_kernel_start() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// G lanes per row (32 / G rows per warp): lane t of a group takes partials t, t + G, ... in ascending
+// order, then a fixed xor-shuffle tree combines the G lanes.  The order never depends on timing:
+// bit-identical results from run to run.
+// Every thread of the warp calls this (the shuffles are warp-wide); `row` is the lane group's row, `row_ok`
+// whether it exists.  The pairs may have been written by other SMs during this same kernel: they are read from L2.
+template <int G>
+__device__ __forceinline__ void merge_rows(const Params& p, long long row, bool row_ok) {
+  const int lane = threadIdx.x & 31, sub = lane % G;
+  const float2* src = reinterpret_cast<const float2*>(p.parts) + (row_ok ? row : 0) * p.parts_per_row;
+  if (p.reduce == FGR_RED_MEANVAR) {
+    // pairs are (mean, sum of squared deviations) of a slot; the slot's column count follows from the
+    // tiling.  Pairwise update: delta = mean_b - mean_a; mean += delta n_b / n; M2 += M2_b + delta^2 n_a n_b / n
+    float n = 0.0f, mean = 0.0f, m2 = 0.0f;
+    for (int t = sub; t < p.parts_per_row; t += G) {
+      const float nb = (float)slot_columns(t, p.N, p.tile_n, p.half_n, p.slots_per_tile);
+      if (nb > 0.0f) {
+        const float2 v = __ldcg(src + t);
+        const float tot = n + nb, delta = v.x - mean;
+        mean += delta * (nb / tot);
+        m2 += v.y + delta * delta * (n * nb / tot);
+        n = tot;
+      }
+    }
+#pragma unroll
+    for (int o = G / 2; o >= 1; o >>= 1) {
+      const float on = __shfl_xor_sync(0xffffffffu, n, o), om = __shfl_xor_sync(0xffffffffu, mean, o),
+                  o2 = __shfl_xor_sync(0xffffffffu, m2, o);
+      // the lower lane's triple is always the left operand, so both lanes compute the same bits
+      const bool hi = (lane & o) != 0;
+      const float na = hi ? on : n, ma = hi ? om : mean, qa = hi ? o2 : m2;
+      const float nb = hi ? n : on, mb = hi ? mean : om, qb = hi ? m2 : o2;
+      const float tot = na + nb;
+      if (tot > 0.0f) {
+        const float delta = mb - ma;
+        mean = ma + delta * (nb / tot);
+        m2 = qa + qb + delta * delta * (na * nb / tot);
+      }
+      n = tot;
+    }
+    if (sub == 0 && row_ok) reinterpret_cast<float2*>(p.out)[row] = make_float2(mean, m2 / (float)p.N);
+    return;
+  }
+  const bool exp_kind = p.reduce != FGR_RED_MAXSUM;
+  float a = -CUDART_INF_F, b = 0.0f;
+#pragma unroll 4
+  for (int t = sub; t < p.parts_per_row; t += G) {
+    float2 v = __ldcg(src + t);
+    if (exp_kind) {
+      float mn = fmaxf(a, v.x);
+      if (mn > -CUDART_INF_F) b = b * expf(a - mn) + v.y * expf(v.x - mn);
+      a = mn;
+    } else {
+      a = fmaxf(a, v.x);
+      b += v.y;
+    }
+  }
+#pragma unroll
+  for (int o = G / 2; o >= 1; o >>= 1) {
+    float oa = __shfl_xor_sync(0xffffffffu, a, o), ob = __shfl_xor_sync(0xffffffffu, b, o);
+    if (exp_kind) {
+      float mn = fmaxf(a, oa);
+      // both operands of the sum are evaluated in the same (lower lane first) order on both lanes
+      float lo_a = (lane & o) ? oa : a, lo_b = (lane & o) ? ob : b;
+      float hi_a = (lane & o) ? a : oa, hi_b = (lane & o) ? b : ob;
+      b = (mn > -CUDART_INF_F) ? lo_b * expf(lo_a - mn) + hi_b * expf(hi_a - mn) : 0.0f;
+      a = mn;
+    } else {
+      float lo_b = (lane & o) ? ob : b, hi_b = (lane & o) ? b : ob;
+      a = fmaxf(a, oa);
+      b = lo_b + hi_b;
+    }
+  }
+  if (sub == 0 && row_ok) {
+    if (p.reduce == FGR_RED_LSE) p.out[row] = a + logf(b);
+    else if (p.reduce != FGR_RED_SOFTMAX) reinterpret_cast<float2*>(p.out)[row] = make_float2(a, b);
+  }
+}
+
+// Lanes per row of the merge: few, each folding up to eight pairs (its loads are independent and go out together).
+__host__ __device__ inline int merge_lanes(int parts_per_row) { return parts_per_row <= 8 ? 2 : parts_per_row <= 64 ? 8 : 32; }
+
 template <typename T>
 __global__ void __launch_bounds__(256) simt_gemm_kernel(const Params p) {
   __shared__ __align__(16) float Xs[BK][kSimtTile + PAD];
@@ -82,21 +171,30 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(const Params p) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
 
-  // the loads of k-block i + 1 are issued before the FMAs of k-block i, so their latency is hidden
-  auto fetch = [&](int k0, float4& xv, float4& wv) {
-    xv = make_float4(0.f, 0.f, 0.f, 0.f);
-    wv = xv;
-    if (k0 + lk < p.K) {   // K is a multiple of 4: the four elements are in range together
-      if (m0 + lr < p.M) xv = load4(X + (long long)(m0 + lr) * p.ldx + k0 + lk);
-      if (n0 + lr < p.N) wv = load4(W + (long long)(n0 + lr) * p.ldw + k0 + lk);
+  // the loads of k-block i + 1 are issued before the FMAs of k-block i, so their latency is hidden; a k-block
+  // is 32 wide (two 16-byte loads per thread and matrix), which halves the number of load -> barrier -> FMA
+  // rounds a short problem is bound by
+  auto fetch = [&](int k0, float4 (&xv)[2], float4 (&wv)[2]) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      xv[h] = make_float4(0.f, 0.f, 0.f, 0.f);
+      wv[h] = xv[h];
+      if (k0 + 16 * h + lk < p.K) {   // K is a multiple of 4: the four elements are in range together
+        if (m0 + lr < p.M) xv[h] = load4(X + (long long)(m0 + lr) * p.ldx + k0 + 16 * h + lk);
+        if (n0 + lr < p.N) wv[h] = load4(W + (long long)(n0 + lr) * p.ldw + k0 + 16 * h + lk);
+      }
     }
   };
-  float4 xv, wv;
+  float4 xv[2], wv[2];
   fetch(0, xv, wv);
   for (int k0 = 0; k0 < p.K; k0 += BK) {
     __syncthreads();
-    Xs[lk + 0][lr] = xv.x; Xs[lk + 1][lr] = xv.y; Xs[lk + 2][lr] = xv.z; Xs[lk + 3][lr] = xv.w;
-    Ws[lk + 0][lr] = wv.x; Ws[lk + 1][lr] = wv.y; Ws[lk + 2][lr] = wv.z; Ws[lk + 3][lr] = wv.w;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int kk = 16 * h + lk;
+      Xs[kk + 0][lr] = xv[h].x; Xs[kk + 1][lr] = xv[h].y; Xs[kk + 2][lr] = xv[h].z; Xs[kk + 3][lr] = xv[h].w;
+      Ws[kk + 0][lr] = wv[h].x; Ws[kk + 1][lr] = wv[h].y; Ws[kk + 2][lr] = wv[h].z; Ws[kk + 3][lr] = wv[h].w;
+    }
     __syncthreads();
     if (k0 + BK < p.K) fetch(k0 + BK, xv, wv);
 #pragma unroll
@@ -175,92 +273,31 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(const Params p) {
       *dst = make_float2(mx, second);
     }
   }
-}
-
-// Programmatic dependent launch: the kernels below may be made resident while the kernel before
-// them in the stream is still running; this wait returns once that kernel has completed and its
-// writes are visible.  (A no-op for a kernel launched the ordinary way.)
-__device__ __forceinline__ void wait_for_prior_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-// Lets the next kernel in the stream (if it was launched as a programmatic dependent) become
-// resident now and run its set-up; it still waits for this grid to finish before touching memory.
-__device__ __forceinline__ void let_next_kernel_start() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-
-// G lanes per row (32 / G rows per warp): lane t of a group takes partials t, t + G, ... in ascending
-// order, then a fixed xor-shuffle tree combines the G lanes.  The order never depends on timing:
-// bit-identical results from run to run.
-template <int G>
-__device__ __forceinline__ void merge_rows(const Params& p, long long block) {
-  const int lane = threadIdx.x & 31, sub = lane % G;
-  const long long warp = block * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const long long row = warp * (32 / G) + lane / G;
-  const bool row_ok = row < (long long)p.batch * p.M;
-  const float2* src = reinterpret_cast<const float2*>(p.parts) + (row_ok ? row : 0) * p.parts_per_row;
-  if (p.reduce == FGR_RED_MEANVAR) {
-    // pairs are (mean, sum of squared deviations) of a slot; the slot's column count follows from the
-    // tiling.  Pairwise update: delta = mean_b - mean_a; mean += delta n_b / n; M2 += M2_b + delta^2 n_a n_b / n
-    float n = 0.0f, mean = 0.0f, m2 = 0.0f;
-    for (int t = sub; t < p.parts_per_row; t += G) {
-      const float nb = (float)slot_columns(t, p.N, p.tile_n, p.half_n, p.slots_per_tile);
-      if (nb > 0.0f) {
-        const float2 v = src[t];
-        const float tot = n + nb, delta = v.x - mean;
-        mean += delta * (nb / tot);
-        m2 += v.y + delta * delta * (n * nb / tot);
-        n = tot;
+  // ---- split-N merge without a second launch (p.done != null: every reduction but softmax, whose second
+  // pass rewrites P).  The CTAs of a block of 64 rows count themselves; the one that brings the count to the
+  // number of column tiles knows that all partial pairs of those rows are in memory and merges them, exactly
+  // as the merge kernel would (same lanes per row, same order: the same bits), then zeroes the count for the
+  // next run.  No CTA waits for another.  Small problems are bound by launch latency: this halves it.
+  if (p.done) {
+    __shared__ int last;
+    __threadfence();                       // this thread's pairs before the count
+    __syncthreads();
+    unsigned int* count = p.done + (long long)bt * gridDim.y + blockIdx.y;
+    if (t == 0) last = atomicAdd(count, 1u) + 1 == gridDim.x ? 1 : 0;
+    __syncthreads();
+    if (last) {
+      if (t == 0) *count = 0u;
+      __threadfence();                     // the other CTAs' pairs, ordered after the count that revealed them
+      const int g = merge_lanes(p.parts_per_row);
+      for (int first = 0; first < kSimtTile; first += 256 / g) {
+        const int li = first + t / g;      // row of the tile this lane group takes in this pass
+        const bool ok = li < kSimtTile && m0 + li < p.M;
+        const long long row = (long long)bt * p.M + m0 + li;
+        if (g == 2) merge_rows<2>(p, row, ok);
+        else if (g == 8) merge_rows<8>(p, row, ok);
+        else merge_rows<32>(p, row, ok);
       }
     }
-#pragma unroll
-    for (int o = G / 2; o >= 1; o >>= 1) {
-      const float on = __shfl_xor_sync(0xffffffffu, n, o), om = __shfl_xor_sync(0xffffffffu, mean, o),
-                  o2 = __shfl_xor_sync(0xffffffffu, m2, o);
-      // the lower lane's triple is always the left operand, so both lanes compute the same bits
-      const bool hi = (lane & o) != 0;
-      const float na = hi ? on : n, ma = hi ? om : mean, qa = hi ? o2 : m2;
-      const float nb = hi ? n : on, mb = hi ? mean : om, qb = hi ? m2 : o2;
-      const float tot = na + nb;
-      if (tot > 0.0f) {
-        const float delta = mb - ma;
-        mean = ma + delta * (nb / tot);
-        m2 = qa + qb + delta * delta * (na * nb / tot);
-      }
-      n = tot;
-    }
-    if (sub == 0 && row_ok) reinterpret_cast<float2*>(p.out)[row] = make_float2(mean, m2 / (float)p.N);
-    return;
-  }
-  const bool exp_kind = p.reduce != FGR_RED_MAXSUM;
-  float a = -CUDART_INF_F, b = 0.0f;
-#pragma unroll 4
-  for (int t = sub; t < p.parts_per_row; t += G) {
-    float2 v = src[t];
-    if (exp_kind) {
-      float mn = fmaxf(a, v.x);
-      if (mn > -CUDART_INF_F) b = b * expf(a - mn) + v.y * expf(v.x - mn);
-      a = mn;
-    } else {
-      a = fmaxf(a, v.x);
-      b += v.y;
-    }
-  }
-#pragma unroll
-  for (int o = G / 2; o >= 1; o >>= 1) {
-    float oa = __shfl_xor_sync(0xffffffffu, a, o), ob = __shfl_xor_sync(0xffffffffu, b, o);
-    if (exp_kind) {
-      float mn = fmaxf(a, oa);
-      // both operands of the sum are evaluated in the same (lower lane first) order on both lanes
-      float lo_a = (lane & o) ? oa : a, lo_b = (lane & o) ? ob : b;
-      float hi_a = (lane & o) ? a : oa, hi_b = (lane & o) ? b : ob;
-      b = (mn > -CUDART_INF_F) ? lo_b * expf(lo_a - mn) + hi_b * expf(hi_a - mn) : 0.0f;
-      a = mn;
-    } else {
-      float lo_b = (lane & o) ? ob : b, hi_b = (lane & o) ? b : ob;
-      a = fmaxf(a, oa);
-      b = lo_b + hi_b;
-    }
-  }
-  if (sub == 0 && row_ok) {
-    if (p.reduce == FGR_RED_LSE) p.out[row] = a + logf(b);
-    else if (p.reduce != FGR_RED_SOFTMAX) reinterpret_cast<float2*>(p.out)[row] = make_float2(a, b);
   }
 }
 
@@ -268,7 +305,8 @@ template <int G>
 __global__ void __launch_bounds__(256) merge_kernel(const Params p) {
   let_next_kernel_start();
   wait_for_prior_kernel();
-  merge_rows<G>(p, blockIdx.x);
+  const long long row = ((long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * (32 / G) + (threadIdx.x & 31) / G;
+  merge_rows<G>(p, row, row < (long long)p.batch * p.M);
 }
 
 // Softmax, second pass.  The GEMM pass stored E[m, n] = exp(y - m_slot) per partial slot together
@@ -564,8 +602,9 @@ cudaError_t launch_merge(const Params& p, cudaStream_t stream) {
   // the grid stays small.  The next run's main kernel, a programmatic dependent of this one, may move in only
   // once every CTA here has started; a grid that fits beside the main kernel in one wave (two CTAs per SM) lets
   // it do so while the main kernel's CTAs are still leaving.
-  if (p.parts_per_row <= 8) return launch_dependent(merge_kernel<2>, (unsigned)((rows + 127) / 128), 256, 0, stream, p);
-  if (p.parts_per_row <= 64) return launch_dependent(merge_kernel<8>, (unsigned)((rows + 31) / 32), 256, 0, stream, p);
+  const int g = merge_lanes(p.parts_per_row);
+  if (g == 2) return launch_dependent(merge_kernel<2>, (unsigned)((rows + 127) / 128), 256, 0, stream, p);
+  if (g == 8) return launch_dependent(merge_kernel<8>, (unsigned)((rows + 31) / 32), 256, 0, stream, p);
   return launch_dependent(merge_kernel<32>, (unsigned)((rows + 7) / 8), 256, 0, stream, p);
 }
 
