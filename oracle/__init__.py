@@ -173,6 +173,37 @@ def conv1d_windows(x, taps: int, stride: int = 1):
     return A
 
 
+def conv2d_windows(x, R: int, S: int):
+    """Rows of the 2-D convolution written out as a matrix (no arithmetic, only copies).
+
+    The operator category "convolution" (Section 1; Section 4.1, Datasets) in its image form: for a
+    channels-last input x [batch, H, Wd, C] and a filter bank w [N, R, S, C] (no padding, stride 1, no dilation),
+
+        z[b, p, q, n] = sum_{r < R} sum_{s < S} sum_{c < C} x[b, p + r, q + s, c] * w[n, r, s, c],
+        p = 0 .. H - R,  q = 0 .. Wd - S,
+
+    which is the product of the window matrix  A[b, p Q + q, (r S + s) C + c] = x[b, p + r, q + s, c]
+    (Q = Wd - S + 1) with  w  viewed as [N, R * S * C].  Returns A [batch, P * Q, R * S * C]; ``run`` on (A, w)
+    is then the definition of the fused convolution + epilogue + reduction over the output channels.
+    """
+    x = np.ascontiguousarray(x)
+    if x.ndim == 3:
+        x = x[None]
+    batch, H, Wd, C = x.shape
+    if R < 1 or R > H or S < 1 or S > Wd:
+        raise ValueError("the filter must fit inside the image")
+    P, Q = H - R + 1, Wd - S + 1
+    A = np.empty((batch, P * Q, R * S * C), dtype=x.dtype)
+    for b in range(batch):
+        for pp in range(P):
+            for q in range(Q):
+                for r in range(R):
+                    for t in range(S):
+                        k = (r * S + t) * C
+                        A[b, pp * Q + q, k:k + C] = x[b, pp + r, q + t, :]
+    return A
+
+
 def run_problem(p, rows=None, want_y=True, nthreads=0):
     """``run`` on an object carrying X, W, bias, scale_vec and the descriptor fields as attributes.
     With ``p.conv_taps > 1``, ``p.X`` is the channels-last input [batch, L, C] of a 1-D convolution and

@@ -430,6 +430,54 @@ def test_conv1d_matches_library_fp64_and_shift_kernel():
     np.testing.assert_array_equal(Yd.ravel(), x[0, r0:r0 + L - R + 1, c0].astype(np.float64))
 
 
+# ---------------------------------------------------------------- 2-D convolution as window matrix
+def test_conv2d_windows_hand_example():
+    # one channel, a 3 x 3 image 1..9, a 2 x 2 filter: four windows, each (top-left, top-right, bottom-left, bottom-right)
+    x = np.arange(1, 10, dtype=np.float32).reshape(1, 3, 3, 1)
+    A = oracle.conv2d_windows(x, 2, 2)
+    assert A.shape == (1, 4, 4)
+    np.testing.assert_array_equal(A[0], [[1, 2, 4, 5], [2, 3, 5, 6], [4, 5, 7, 8], [5, 6, 8, 9]])
+    # the filter ((1, 0), (0, -1)) gives top-left minus bottom-right: 1-5, 2-6, 4-8, 5-9
+    w = np.array([1, 0, 0, -1], dtype=np.float32).reshape(1, 1, 4)
+    Y, _, _ = _run(A, w, None, None, reduce=oracle.RED_MAXSUM)
+    np.testing.assert_array_equal(Y.ravel(), [-4, -4, -4, -4])
+    # two channels interleave per pixel: window (p, q) = pixels (p,q) (p,q+1) (p+1,q) (p+1,q+1), channels inside
+    x2 = np.stack([x[..., 0], 10 * x[..., 0]], -1)
+    np.testing.assert_array_equal(oracle.conv2d_windows(x2, 2, 2)[0, 3], [5, 50, 6, 60, 8, 80, 9, 90])
+    # a 1 x 1 filter is the plain linear layer on the pixels; a filter of the image's size gives one window
+    np.testing.assert_array_equal(oracle.conv2d_windows(x2, 1, 1)[0], x2.reshape(9, 2))
+    np.testing.assert_array_equal(oracle.conv2d_windows(x2, 3, 3)[0], x2.reshape(1, 18))
+    with pytest.raises(ValueError):
+        oracle.conv2d_windows(x, 4, 1)
+
+
+def test_conv2d_reduces_to_conv1d_and_matches_library_fp64():
+    B, H, Wd, C, N, R, S = 2, 7, 9, 4, 5, 3, 2
+    x = _rand((B, H, Wd, C), 61)
+    w = _rand((N, R, S, C), 62, tid=8)
+    b = gi.uniform(63, 3, N, -1, 1)
+    A = oracle.conv2d_windows(x, R, S)
+    P, Q = H - R + 1, Wd - S + 1
+    assert A.shape == (B, P * Q, R * S * C)
+    # one filter row (R = 1): every image row is a 1-D convolution of its own
+    A1 = oracle.conv2d_windows(x, 1, S)
+    for h in range(H):
+        np.testing.assert_array_equal(A1[:, h * Q:(h + 1) * Q], oracle.conv1d_windows(x[:, h], S))
+    Y, out, _ = oracle.run(A, np.broadcast_to(w.reshape(1, N, R * S * C), (B, N, R * S * C)).copy(), b, None, dtype=oracle.F32,
+                           act=oracle.ACT_RELU, scale_kind=oracle.SCALE_NONE, reduce=oracle.RED_LSE)
+    # library routine: torch's conv2d takes [B, C, H, W] and weights [N, C, R, S]
+    ref = torch.nn.functional.conv2d(torch.from_numpy(x).double().permute(0, 3, 1, 2), torch.from_numpy(w).double().permute(0, 3, 1, 2),
+                                     torch.from_numpy(b).double()).relu().permute(0, 2, 3, 1).reshape(B * P * Q, N)
+    np.testing.assert_allclose(Y, ref.numpy(), rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(out[:, 0], torch.logsumexp(ref, 1).numpy(), rtol=1e-13)
+    # a filter that is 1 at (r0, s0, c0) and 0 elsewhere copies the shifted image: z[b, p, q] = x[b, p + r0, q + s0, c0]
+    r0, s0, c0 = 2, 1, 3
+    d = np.zeros((1, 1, R * S * C), np.float32)
+    d[0, 0, (r0 * S + s0) * C + c0] = 1.0
+    Yd, _, _ = oracle.run(A[:1], d, None, None, dtype=oracle.F32, act=oracle.ACT_NONE, scale_kind=oracle.SCALE_NONE, reduce=oracle.RED_MAXSUM)
+    np.testing.assert_array_equal(Yd.reshape(P, Q), x[0, r0:r0 + P, s0:s0 + Q, c0].astype(np.float64))
+
+
 # ---------------------------------------------------------------- mean / variance over N
 def test_meanvar_closed_forms():
     N = 12
