@@ -173,7 +173,10 @@ FGR_API int fgr_get_plan(const fgr_handle* h, fgr_plan_info* info /*host, out*/)
 
 /*
  * fgr_run: enqueues the whole operator (GEMM mainloop, fused epilogue, per-tile row reduction,
- * split-N merge, softmax normalisation) on `cuda_stream` and returns without synchronising.
+ * split-N merge, softmax normalisation) on `cuda_stream` and returns without synchronising.  It launches
+ * one to four kernels (fgr_plan_info.launches); on the tensor-core paths the softmax normalisation kernel
+ * runs beside the main kernel and follows it block of rows by block of rows (the main kernel never waits for
+ * it); all of them are complete, in stream order, before anything enqueued after fgr_run starts.
  *   X, W       device, dtype, read-only
  *   bias       device fp32 [N] (or [batch, N]); NULL = no bias
  *   scale_vec  device fp32 [N]; required iff scale_kind == FGR_SCALE_PER_COLUMN
@@ -197,7 +200,10 @@ FGR_API int fgr_run(fgr_handle* h, const void* X, const void* W, const float* bi
  * descriptor says).  Copies the inputs to device staging buffers owned by the handle (allocated on
  * the first call, freed by fgr_destroy), runs, copies Y / out back and synchronises before
  * returning.  Returns the device status as fgr_get_status would.  Pinned host memory makes the
- * copies asynchronous and faster but is not required.
+ * copies asynchronous and faster but is not required.  Problems of at least four batches, or of one batch
+ * and at least 1024 rows (plain GEMMs), are run as four chunks - blocks of batches or of rows, which are
+ * independent - on three streams, so that the copy in of one chunk, the kernels of the previous one and
+ * the copy out of the one before overlap; the results are those of the whole problem.
  */
 FGR_API int fgr_run_host(fgr_handle* h, const void* X, const void* W, const float* bias, const float* scale_vec,
                  void* Y, float* out);
