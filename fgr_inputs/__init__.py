@@ -133,6 +133,8 @@ class Problem:
     w_shared: int = 0      # 1: W is [1, N, K], one matrix for every batch element
     conv_taps: int = 0     # R > 1: 1-D convolution; X is then [batch, (M - 1) * stride + R, K / R] (channels last)
     conv_stride: int = 1
+    conv_rows: int = 0     # R > 1: 2-D convolution; X is then the image [batch, H, conv_width, K / (R * S)], S = max(conv_taps, 1),
+    conv_width: int = 0    # and M = (P - 1) * conv_width + Q output rows at the image's row pitch (P = H - R + 1, Q = conv_width - S + 1)
     X: np.ndarray | None = None
     W: np.ndarray | None = None
     bias: np.ndarray | None = None
@@ -157,6 +159,9 @@ class Problem:
         e = self.elem_bytes
         taps = max(self.conv_taps, 1)
         x_elems = (self.M - 1) * min(self.conv_stride * (self.K // taps), self.K) + self.K if taps > 1 else self.M * self.K
+        if self.conv_rows > 1:     # the pixels the M windows cover
+            c = self.K // (self.conv_rows * taps)
+            x_elems = (self.M - 1 + (self.conv_rows - 1) * self.conv_width) * c + taps * c
         b = (self.batch * x_elems + (1 if self.w_shared else self.batch) * self.N * self.K) * e
         if self.bias is not None:
             b += self.bias.size * 4
@@ -176,7 +181,8 @@ def _store(a: np.ndarray, dtype: int) -> np.ndarray:
 
 def make_problem(name, batch, M, N, K, dtype, act, scale_kind, reduce, *, scale=1.0, write_y=0,
                  x_std=None, w_std=None, bias_range=(-0.1, 0.1), scale_range=(0.5, 1.5),
-                 bias_per_batch=0, seed=0, materialize=True, conv_taps=0, w_shared=0, residual_std=None, conv_stride=1) -> Problem:
+                 bias_per_batch=0, seed=0, materialize=True, conv_taps=0, w_shared=0, residual_std=None, conv_stride=1,
+                 conv_rows=0, conv_width=0) -> Problem:
     """Draws a problem with the value distributions of the named workloads.
 
     x_std / w_std default to 1/sqrt(K); bias ~ U(bias_range) (None -> no bias);
@@ -186,6 +192,7 @@ def make_problem(name, batch, M, N, K, dtype, act, scale_kind, reduce, *, scale=
     w_std = 1.0 / math.sqrt(K) if w_std is None else w_std
     p = Problem(name, batch, M, N, K, dtype, act, scale_kind, reduce, scale=float(scale),
                 write_y=write_y, bias_per_batch=bias_per_batch, conv_taps=conv_taps, w_shared=w_shared, conv_stride=conv_stride,
+                conv_rows=conv_rows, conv_width=conv_width,
                 recipe=dict(seed=seed, x_std=x_std, w_std=w_std, bias_range=bias_range,
                             scale_range=scale_range if scale_kind == SCALE_PER_COLUMN else None))
     if not materialize:
@@ -194,7 +201,14 @@ def make_problem(name, batch, M, N, K, dtype, act, scale_kind, reduce, *, scale=
         if scale_kind == SCALE_PER_COLUMN:
             p.scale_vec = np.empty(N, dtype=np.float32)
         return p
-    if conv_taps > 1:      # the input signal itself; the operator reads overlapping windows of it
+    if conv_rows > 1:      # the image itself: M = (P - 1) * conv_width + Q output rows need H = P + conv_rows - 1 image rows
+        S = max(conv_taps, 1)
+        Q = conv_width - S + 1
+        if (M - Q) % conv_width != 0 or M < Q:
+            raise ValueError("M must be (P - 1) * conv_width + Q for a whole number P of output rows")
+        H, C = (M - Q) // conv_width + conv_rows, K // (conv_rows * S)
+        p.X = _store(normal(seed, TENSOR_X, batch * H * conv_width * C, x_std), dtype).reshape(batch, H, conv_width, C)
+    elif conv_taps > 1:    # the input signal itself; the operator reads overlapping windows of it
         L, C = (M - 1) * conv_stride + conv_taps, K // conv_taps
         p.X = _store(normal(seed, TENSOR_X, batch * L * C, x_std), dtype).reshape(batch, L, C)
     else:

@@ -122,6 +122,21 @@ typedef struct fgr_desc {
   int32_t w_shared;        /* 0: W is [batch, N, K] (one weight matrix per batch element).  1: W is one [N, K] matrix
                               used by every batch element (bsw is ignored) - a filter bank shared by all signals of
                               a convolution, or one linear layer applied to a batch of inputs */
+  int32_t conv_rows;       /* 0 or 1: not a 2-D convolution.  R > 1: 2-D convolution as an implicit GEMM (the operator
+                              category "convolution", Section 1 and Section 4.1), stride 1, no padding, no dilation:
+                              X is the channels-last image [batch, H, conv_width, C], W the filters [N, R, S, C] with
+                              S = conv_taps (0 or 1 mean S = 1) and C = K / (R * S),
+                                z[b, p, q, n] = sum_r sum_s sum_c X[b, p + r, q + s, c] * W[n, r, s, c].
+                              The output keeps the image's row pitch: GEMM row m = p * conv_width + q, so Y is
+                              [batch, P, conv_width, N] seen as [batch, M, N] with M = (P - 1) * conv_width + Q rows
+                              (P = H - R + 1, Q = conv_width - S + 1), and so is `out`.  Rows with q >= Q are not outputs
+                              of the convolution (their windows wrap into the next image row): they hold finite
+                              values of no meaning and the caller skips them.  Nothing is copied or unfolded: filter
+                              row r of output row m reads the S * C contiguous elements at X[b, (m + r * conv_width), 0].
+                              ldx must be 0 (= C); bsx defaults to the smallest image that holds the M windows; the
+                              image must hold (M - 1 + (R - 1) * conv_width + S) pixels.  Needs w_shared = 1 or batch = 1;
+                              bf16 on the tiled / streaming tensor-core paths, fp32 (and bf16) on the CUDA-core path. */
+  int32_t conv_width;      /* image row length in pixels when conv_rows > 1 (>= S) */
 } fgr_desc;
 
 /* What fgr_plan / fgr_create decided; plain host data, for callers, tests and benchmarks. */

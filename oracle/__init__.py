@@ -208,6 +208,11 @@ def run_problem(p, rows=None, want_y=True, nthreads=0):
     """``run`` on an object carrying X, W, bias, scale_vec and the descriptor fields as attributes.
     With ``p.conv_taps > 1``, ``p.X`` is the channels-last input [batch, L, C] of a 1-D convolution and
     ``p.W`` its filters [batch, N, taps * C]."""
+    if getattr(p, "conv_rows", 0) > 1:
+        # rows are then indexed over the convolution's own outputs, [batch, P, Q] flattened (no image row pitch)
+        return run(conv2d_windows(p.X, p.conv_rows, max(p.conv_taps, 1)), p.W, p.bias, p.scale_vec, dtype=p.dtype, act=p.act,
+                   scale_kind=p.scale_kind, reduce=p.reduce, scale=p.scale, bias_per_batch=p.bias_per_batch,
+                   rows=rows, want_y=want_y, nthreads=nthreads, residual=getattr(p, "residual", None))
     if getattr(p, "conv_taps", 0) > 1:
         return run(conv1d_windows(p.X, p.conv_taps, getattr(p, "conv_stride", 1) or 1), p.W, p.bias, p.scale_vec, dtype=p.dtype, act=p.act,
                    scale_kind=p.scale_kind, reduce=p.reduce, scale=p.scale, bias_per_batch=p.bias_per_batch,

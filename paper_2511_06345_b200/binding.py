@@ -38,7 +38,8 @@ class fgr_desc(ctypes.Structure):
                 ("bias_per_batch", ctypes.c_int32), ("device", ctypes.c_int32),
                 ("force_path", ctypes.c_int32), ("force_tile_n", ctypes.c_int32),
                 ("force_cta_pair", ctypes.c_int32), ("force_ksub", ctypes.c_int32),
-                ("conv_taps", ctypes.c_int32), ("w_shared", ctypes.c_int32)]
+                ("conv_taps", ctypes.c_int32), ("w_shared", ctypes.c_int32),
+                ("conv_rows", ctypes.c_int32), ("conv_width", ctypes.c_int32)]
 
 
 class fgr_reduce_desc(ctypes.Structure):
@@ -106,9 +107,10 @@ def lib() -> ctypes.CDLL:
 
 def make_desc(batch, M, N, K, dtype, act, scale_kind, reduce, *, scale=1.0, write_y=0, ldx=0, ldw=0, ldy=0,
               bsx=0, bsw=0, bsy=0, bias_per_batch=0, device=0, force_path=FGR_PATH_AUTO, force_tile_n=0, force_cta_pair=0, force_ksub=0,
-              conv_taps=0, w_shared=0) -> fgr_desc:
+              conv_taps=0, w_shared=0, conv_rows=0, conv_width=0) -> fgr_desc:
     return fgr_desc(ctypes.sizeof(fgr_desc), batch, M, N, K, dtype, act, scale_kind, reduce, scale, write_y,
-                    ldx, ldw, ldy, bsx, bsw, bsy, bias_per_batch, device, force_path, force_tile_n, force_cta_pair, force_ksub, conv_taps, w_shared)
+                    ldx, ldw, ldy, bsx, bsw, bsy, bias_per_batch, device, force_path, force_tile_n, force_cta_pair, force_ksub, conv_taps, w_shared,
+                    conv_rows, conv_width)
 
 
 def fgr_status_string(status: int) -> str:

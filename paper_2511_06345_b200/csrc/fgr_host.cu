@@ -92,14 +92,26 @@ int out_width(int reduce) { return reduce == FGR_RED_LSE ? 1 : reduce == FGR_RED
 
 struct Resolved { long long ldx, ldw, ldy, bsx, bsw, bsy; };
 
+// Elements of X that one batch element's M output rows read, first to last (convolutions: the signal or image).
+long long x_span(const fgr_desc& d, long long ldx) {
+  if (d.conv_rows > 1) {
+    const int s = d.conv_taps > 1 ? d.conv_taps : 1;
+    const long long c = d.K / ((long long)d.conv_rows * s);
+    return ((long long)(d.M - 1) + (long long)(d.conv_rows - 1) * d.conv_width) * ldx + s * c;
+  }
+  return (long long)(d.M - 1) * ldx + d.K;
+}
+
 Resolved resolve_strides(const fgr_desc& d) {
   Resolved r;
-  const int taps = d.conv_taps > 1 ? d.conv_taps : 1;   // 1-D convolution: rows of the implicit matrix overlap
+  const int rows2d = d.conv_rows > 1 ? d.conv_rows : 1;   // 2-D convolution: K is rows2d segments of taps * C elements
+  const int taps = (d.conv_taps > 1 ? d.conv_taps : 1) * rows2d;   // convolution: rows of the implicit matrix overlap
   r.ldx = d.ldx ? d.ldx : d.K / taps;
   r.ldw = d.ldw ? d.ldw : d.K;
   r.ldy = d.ldy ? d.ldy : d.N;
-  // (a strided convolution has ldx = stride * C: its signal is (M - 1) * stride + taps samples of C channels)
-  r.bsx = d.bsx ? d.bsx : (taps > 1 ? (long long)(d.M - 1) * r.ldx + d.K : (long long)d.M * r.ldx);
+  // (a strided 1-D convolution has ldx = stride * C: its signal is (M - 1) * stride + taps samples of C channels;
+  //  a 2-D one reads, for its last output row, up to filter row R - 1 below it: see x_span)
+  r.bsx = d.bsx ? d.bsx : (taps > 1 ? x_span(d, r.ldx) : (long long)d.M * r.ldx);
   r.bsw = d.w_shared ? 0 : (d.bsw ? d.bsw : (long long)d.N * r.ldw);   // shared W: every batch reads the same matrix
   r.bsy = d.bsy ? d.bsy : (long long)d.M * r.ldy;
   return r;
@@ -122,15 +134,23 @@ int validate(const fgr_desc* d) {
   const int g = 16 / elem_bytes(d->dtype);   // elements per 16 bytes
   if (d->K % g || d->N % g) return FGR_ERR_UNSUPPORTED;
   if (d->conv_taps < 0 || (d->w_shared != 0 && d->w_shared != 1)) return FGR_ERR_INVALID_ARG;
-  const int taps = d->conv_taps > 1 ? d->conv_taps : 1;
+  if (d->conv_rows < 0 || d->conv_width < 0) return FGR_ERR_INVALID_ARG;
+  const bool conv2d = d->conv_rows > 1;
+  const int taps = (d->conv_taps > 1 ? d->conv_taps : 1) * (conv2d ? d->conv_rows : 1);
   if (d->K % taps) return FGR_ERR_INVALID_ARG;
   if ((d->K / taps) % g) return FGR_ERR_UNSUPPORTED;
+  if (conv2d) {
+    if (d->conv_width < (d->conv_taps > 1 ? d->conv_taps : 1)) return FGR_ERR_INVALID_ARG;
+    if (d->ldx != 0 && d->ldx != d->K / taps) return FGR_ERR_UNSUPPORTED;   // stride 1 only
+    if (!d->w_shared && d->batch > 1) return FGR_ERR_UNSUPPORTED;            // one filter bank (the W tensor map is [S C, R, N])
+    if (d->ldw != 0 && d->ldw != d->K) return FGR_ERR_UNSUPPORTED;
+  }
   const Resolved r = resolve_strides(*d);
   if (r.ldx < d->K / taps || r.ldw < d->K || r.ldy < d->N) return FGR_ERR_INVALID_ARG;
   // a window must be K contiguous elements: the row stride is the convolution's stride times C, never a padded C
   if (taps > 1 && r.ldx % (d->K / taps) != 0) return FGR_ERR_UNSUPPORTED;
   if (r.ldx % g || r.ldw % g || r.ldy % g || r.bsx % g || r.bsw % g || r.bsy % g) return FGR_ERR_UNSUPPORTED;
-  if (d->batch > 1 && (r.bsx < (long long)(d->M - 1) * r.ldx + d->K || (!d->w_shared && r.bsw < (long long)(d->N - 1) * r.ldw + d->K) ||
+  if (d->batch > 1 && (r.bsx < x_span(*d, r.ldx) || (!d->w_shared && r.bsw < (long long)(d->N - 1) * r.ldw + d->K) ||
                        r.bsy < (long long)(d->M - 1) * r.ldy + d->N))
     return FGR_ERR_INVALID_ARG;
   if ((long long)d->batch * d->M > (1LL << 31) - 1) return FGR_ERR_UNSUPPORTED;
@@ -142,9 +162,10 @@ int validate(const fgr_desc* d) {
 
 double min_bytes(const fgr_desc& d) {
   const double e = elem_bytes(d.dtype);
-  const int taps = d.conv_taps > 1 ? d.conv_taps : 1;   // a convolution's input is read once, not once per tap
+  const int taps = (d.conv_taps > 1 ? d.conv_taps : 1) * (d.conv_rows > 1 ? d.conv_rows : 1);   // a convolution's input is read once, not once per tap
   const Resolved rs = resolve_strides(d);
-  const double x_elems = taps > 1 ? (double)(d.M - 1) * (rs.ldx < d.K ? rs.ldx : d.K) + d.K : (double)d.M * d.K;   // samples actually read
+  const double x_elems = d.conv_rows > 1 ? (double)x_span(d, rs.ldx)
+                         : taps > 1 ? (double)(d.M - 1) * (rs.ldx < d.K ? rs.ldx : d.K) + d.K : (double)d.M * d.K;   // samples actually read
   double b = ((double)d.batch * x_elems + (double)(d.w_shared ? 1 : d.batch) * d.N * d.K) * e;
   b += 4.0 * d.N * (d.bias_per_batch ? d.batch : 1);   // bias (counted whether or not one is passed)
   if (d.scale_kind == FGR_SCALE_PER_COLUMN) b += 4.0 * d.N;
@@ -186,6 +207,12 @@ int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
     else if (d.M <= 128 && pi.flop / pi.min_bytes < kRidgeFlopPerByte) path = FGR_PATH_UMMA_STREAM_W;
     else path = FGR_PATH_UMMA_TILED;
   }
+  const bool conv2d = d.conv_rows > 1;
+  if (conv2d && d.force_path == FGR_PATH_AUTO) {   // 2-D convolution: the tiled / streaming tensor-core paths (bf16) or CUDA cores
+    if (path == FGR_PATH_UMMA_TF32X3) path = FGR_PATH_SIMT;
+    if (path == FGR_PATH_SIMT_GEMV) path = FGR_PATH_UMMA_STREAM_W;
+  }
+  if (conv2d && (path == FGR_PATH_UMMA_TF32X3 || path == FGR_PATH_SIMT_GEMV)) return FGR_ERR_UNSUPPORTED;
   if (path == FGR_PATH_SIMT_GEMV && (d.dtype != FGR_BF16 || d.M > 16 || d.reduce == FGR_RED_SOFTMAX)) return FGR_ERR_UNSUPPORTED;
   if ((path == FGR_PATH_UMMA_TILED || path == FGR_PATH_UMMA_STREAM_W) && d.dtype != FGR_BF16) return FGR_ERR_UNSUPPORTED;
   if (path == FGR_PATH_UMMA_TF32X3 && d.dtype != FGR_F32) return FGR_ERR_UNSUPPORTED;
@@ -197,6 +224,10 @@ int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
   p.dtype = d.dtype; p.act = d.act; p.scale_kind = d.scale_kind; p.reduce = d.reduce;
   p.write_y = d.write_y; p.bias_per_batch = d.bias_per_batch; p.scale = d.scale;
   p.w_shared = d.w_shared;
+  p.conv_rows = conv2d ? d.conv_rows : 0;
+  p.conv_width = d.conv_width;
+  p.conv_kseg = conv2d ? d.K / d.conv_rows : 0;
+  p.kseg_blocks = conv2d ? (p.conv_kseg + kUmmaBlockK - 1) / kUmmaBlockK : 0;
   p.ldx = r.ldx; p.ldw = r.ldw; p.ldy = r.ldy; p.bsx = r.bsx; p.bsw = r.bsw; p.bsy = r.bsy;
 
   if (path == FGR_PATH_SIMT_GEMV) {
@@ -270,6 +301,9 @@ int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
     int ksub = tf32 ? 2 : d.force_ksub;   // 3xTF32: the two sub-blocks of a stage are the hi and lo planes
     if (!ksub) ksub = (d.K > kUmmaBlockK && umma_smem_layout(w_rows, 3, 2).total <= kSmemLimit) ? 2 : 1;
     while (!tf32 && ksub > 1 && umma_smem_layout(w_rows, 2, ksub).total > kSmemLimit) --ksub;
+    if (conv2d) {   // a ring stage must not straddle two filter rows unevenly: whole k-blocks, ksub of them per stage
+      while (ksub > 1 && (d.conv_rows * p.kseg_blocks) % ksub != 0) --ksub;
+    }
     p.ksub = ksub;
     p.k_plane = tf32 ? (d.K + 31) / 32 * 32 : 0;
     p.chunk_blocks = kTf32ChunkBlocks;
@@ -344,14 +378,16 @@ EncodeTiledFn encode_fn() {
 // bf16 [batch, rows, K] with strides (ld, bs) -> 3-D map, box = 64 (K) x box_rows x 1, 128-byte swizzle,
 // out-of-range elements read as zero.
 // (fp32 = true: 4-byte elements, box = 32 (K) x box_rows x 1, the same 128-byte rows.)
+// (box_in_z = true: the box is 64 x 1 x box_rows - rows of the box come from the third dimension, the middle one
+//  selects a plane: the filters of a 2-D convolution as [S C, R, N].)
 int encode_operand(CUtensorMap* map, const void* ptr, int K, int rows, int batch, long long ld, long long bs, int box_rows,
-                   bool fp32 = false) {
+                   bool fp32 = false, bool box_in_z = false) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return FGR_ERR_CUDA;
   const unsigned eb = fp32 ? 4 : 2;
   cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)batch};
-  cuuint64_t strides[2] = {(cuuint64_t)ld * eb, (cuuint64_t)(batch > 1 ? bs : (long long)rows * ld) * eb};
-  cuuint32_t box[3] = {(cuuint32_t)(kUmmaBlockK * 2 / eb), (cuuint32_t)box_rows, 1};
+  cuuint64_t strides[2] = {(cuuint64_t)ld * eb, (cuuint64_t)(batch > 1 || box_in_z ? bs : (long long)rows * ld) * eb};
+  cuuint32_t box[3] = {(cuuint32_t)(kUmmaBlockK * 2 / eb), (cuuint32_t)(box_in_z ? 1 : box_rows), (cuuint32_t)(box_in_z ? box_rows : 1)};
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult rc = fn(map, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -495,14 +531,20 @@ int fgr_run(fgr_handle* h, const void* X, const void* W, const float* bias, cons
       const CUtensorMap* mx = h->maps_x.find(X);
       if (!mx) {
         CUtensorMap* nx = h->maps_x.claim(X);
-        rc = encode_operand(nx, X, d.K, d.M, d.batch, p.ldx, p.bsx, kUmmaTileM);
+        if (p.conv_rows > 1)   // [S C, window rows, batch]: segment r of output row m is window row m + r * conv_width
+          rc = encode_operand(nx, X, p.conv_kseg, d.M + (d.conv_rows - 1) * d.conv_width, d.batch, p.ldx, p.bsx, kUmmaTileM);
+        else
+          rc = encode_operand(nx, X, d.K, d.M, d.batch, p.ldx, p.bsx, kUmmaTileM);
         if (rc != FGR_OK) h->maps_x.forget(X);
         mx = nx;
       }
       const CUtensorMap* mw = rc == FGR_OK ? h->maps_w.find(W) : nullptr;
       if (rc == FGR_OK && !mw) {
         CUtensorMap* nw = h->maps_w.claim(W);
-        rc = encode_operand(nw, W, d.K, d.N, d.w_shared ? 1 : d.batch, p.ldw, p.bsw, p.tile_n / p.cta_pair);
+        if (p.conv_rows > 1)   // [S C, R, N]: one filter bank; filter row r of filter n starts at W[n * K + r * S C]
+          rc = encode_operand(nw, W, p.conv_kseg, d.conv_rows, d.N, p.conv_kseg, p.ldw, p.tile_n / p.cta_pair, false, true);
+        else
+          rc = encode_operand(nw, W, d.K, d.N, d.w_shared ? 1 : d.batch, p.ldw, p.bsw, p.tile_n / p.cta_pair);
         if (rc != FGR_OK) h->maps_w.forget(W);
         mw = nw;
       }
@@ -567,7 +609,7 @@ static bool plan_host_chunks(fgr_handle* h) {
   h->sub_count = 1;
   const fgr_desc& d = h->desc;
   const Params& b = h->base;
-  if (d.conv_taps > 1) return false;   // overlapping rows: the chunks' input copies would overlap too
+  if (d.conv_taps > 1 || d.conv_rows > 1) return false;   // overlapping rows: the chunks' input copies would overlap too
   long long total, unit;
   if (d.batch >= kHostChunks) { h->sub_by_batch = true; total = d.batch; unit = 1; }
   else if (d.batch == 1 && d.M >= kHostChunks * 256) { h->sub_by_batch = false; total = d.M; unit = 256; }
@@ -622,7 +664,7 @@ int fgr_run_host(fgr_handle* h, const void* X, const void* W, const float* bias,
   const size_t e = (size_t)elem_bytes(d.dtype);
   // extents in bytes of each buffer as laid out by the descriptor's strides
   const size_t want[7] = {
-      ((size_t)(d.batch - 1) * b.bsx + (size_t)(d.M - 1) * b.ldx + d.K) * e,
+      ((size_t)(d.batch - 1) * b.bsx + (size_t)x_span(d, b.ldx)) * e,
       ((size_t)(d.batch - 1) * b.bsw + (size_t)(d.N - 1) * b.ldw + d.K) * e,
       bias ? (size_t)d.N * (d.bias_per_batch ? d.batch : 1) * 4 : 0,
       scale_vec ? (size_t)d.N * 4 : 0,

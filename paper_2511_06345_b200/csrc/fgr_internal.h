@@ -43,6 +43,9 @@ struct Params {
   int cta_pair;        // tcgen05 paths: 1 = each CTA works alone, 2 = clusters of two CTAs share 256-row tiles
   int k_plane;         // 3xTF32 path: K rounded up to 32 = width of the hi plane (the lo plane follows it)
   int w_shared;        // 1: W is one [N, K] matrix used by every batch element (bsw = 0)
+  // 2-D convolution (conv_rows > 1): K is conv_rows segments of conv_kseg = S * C contiguous elements; segment r of
+  // output row m starts at X row m + r * conv_width (rows of C elements); a segment is kseg_blocks 64-wide k-blocks
+  int conv_rows, conv_width, conv_kseg, kseg_blocks;
   int chunk_blocks;    // 3xTF32 path: 32-wide k-blocks accumulated in tensor memory before the epilogue adds them up
   // Softmax on the tcgen05 paths: the normalise kernel runs beside the main kernel and rescales a block of rows
   // as soon as all its tiles are stored.  done[u] (in the workspace head) counts the epilogue warps that have

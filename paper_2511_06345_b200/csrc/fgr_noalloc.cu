@@ -46,7 +46,7 @@ int fgr_run_static(const fgr_desc* desc, const void* X, const void* W, const flo
   fgr_plan_info plan;
   int rc = fgr_plan(&d, 0, &plan);
   if (rc != FGR_OK) return rc;
-  if (d.conv_taps > 1) return FGR_ERR_UNSUPPORTED;   // plain GEMMs only
+  if (d.conv_taps > 1 || d.conv_rows > 1) return FGR_ERR_UNSUPPORTED;   // plain GEMMs only
   const unsigned long long need = (unsigned long long)d.batch * d.M * plan.parts_per_row * 8ull;
   if (need > kScratchBytes) return FGR_ERR_WORKSPACE;   // the fixed scratch cannot hold this problem's partial pairs
 

@@ -73,8 +73,15 @@ __device__ __forceinline__ void let_next_kernel_start() { asm volatile("griddepc
 // order, then a fixed xor-shuffle tree combines the G lanes.  The order never depends on timing:
 // bit-identical results from run to run.
 // Every thread of the warp calls this (the shuffles are warp-wide); `row` is the lane group's row, `row_ok`
-// whether it exists.  The pairs may have been written by other SMs during this same kernel: they are read from L2.
-template <int G>
+// whether it exists.  FROM_L2: the pairs may have been written by other SMs during this same kernel, so they
+// are read past L1 (in the merge kernel, a launch of its own, ordinary loads are 1.8 us faster on 128 rows x
+// 256 pairs: 55.0 against 56.9 us for the weight-streaming workload's whole step).
+template <int G, bool FROM_L2>
+__device__ __forceinline__ float2 load_pair(const float2* p) {
+  if constexpr (FROM_L2) return __ldcg(p);
+  else return *p;
+}
+template <int G, bool FROM_L2>
 __device__ __forceinline__ void merge_rows(const Params& p, long long row, bool row_ok) {
   const int lane = threadIdx.x & 31, sub = lane % G;
   const float2* src = reinterpret_cast<const float2*>(p.parts) + (row_ok ? row : 0) * p.parts_per_row;
@@ -85,7 +92,7 @@ __device__ __forceinline__ void merge_rows(const Params& p, long long row, bool 
     for (int t = sub; t < p.parts_per_row; t += G) {
       const float nb = (float)slot_columns(t, p.N, p.tile_n, p.half_n, p.slots_per_tile);
       if (nb > 0.0f) {
-        const float2 v = __ldcg(src + t);
+        const float2 v = load_pair<G, FROM_L2>(src + t);
         const float tot = n + nb, delta = v.x - mean;
         mean += delta * (nb / tot);
         m2 += v.y + delta * delta * (n * nb / tot);
@@ -115,7 +122,7 @@ __device__ __forceinline__ void merge_rows(const Params& p, long long row, bool 
   float a = -CUDART_INF_F, b = 0.0f;
 #pragma unroll 4
   for (int t = sub; t < p.parts_per_row; t += G) {
-    float2 v = __ldcg(src + t);
+    float2 v = load_pair<G, FROM_L2>(src + t);
     if (exp_kind) {
       float mn = fmaxf(a, v.x);
       if (mn > -CUDART_INF_F) b = b * expf(a - mn) + v.y * expf(v.x - mn);
@@ -180,7 +187,11 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(const Params p) {
       xv[h] = make_float4(0.f, 0.f, 0.f, 0.f);
       wv[h] = xv[h];
       if (k0 + 16 * h + lk < p.K) {   // K is a multiple of 4: the four elements are in range together
-        if (m0 + lr < p.M) xv[h] = load4(X + (long long)(m0 + lr) * p.ldx + k0 + 16 * h + lk);
+        // 2-D convolution: element k of the row lies in filter row k / (S C), which reads the image conv_width
+        // pixels further down (S C is a multiple of 4, so the four elements stay in one filter row)
+        const int kk = k0 + 16 * h + lk, fr = p.conv_rows > 1 ? kk / p.conv_kseg : 0;
+        const long long xoff = p.conv_rows > 1 ? (long long)fr * p.conv_width * p.ldx + (kk - fr * p.conv_kseg) : kk;
+        if (m0 + lr < p.M) xv[h] = load4(X + (long long)(m0 + lr) * p.ldx + xoff);
         if (n0 + lr < p.N) wv[h] = load4(W + (long long)(n0 + lr) * p.ldw + k0 + 16 * h + lk);
       }
     }
@@ -293,9 +304,9 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(const Params p) {
         const int li = first + t / g;      // row of the tile this lane group takes in this pass
         const bool ok = li < kSimtTile && m0 + li < p.M;
         const long long row = (long long)bt * p.M + m0 + li;
-        if (g == 2) merge_rows<2>(p, row, ok);
-        else if (g == 8) merge_rows<8>(p, row, ok);
-        else merge_rows<32>(p, row, ok);
+        if (g == 2) merge_rows<2, true>(p, row, ok);
+        else if (g == 8) merge_rows<8, true>(p, row, ok);
+        else merge_rows<32, true>(p, row, ok);
       }
     }
   }
@@ -306,7 +317,7 @@ __global__ void __launch_bounds__(256) merge_kernel(const Params p) {
   let_next_kernel_start();
   wait_for_prior_kernel();
   const long long row = ((long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * (32 / G) + (threadIdx.x & 31) / G;
-  merge_rows<G>(p, row, row < (long long)p.batch * p.M);
+  merge_rows<G, false>(p, row, row < (long long)p.batch * p.M);
 }
 
 // Softmax, second pass.  The GEMM pass stored E[m, n] = exp(y - m_slot) per partial slot together

@@ -406,7 +406,8 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kstep = TF32 ? kUmmaBlockK / 2 : kUmmaBlockK * p.ksub;   // K elements per ring stage (128-byte rows)
-  const int kblocks = (p.K + kstep - 1) / kstep;
+  // (2-D convolution: conv_rows segments of kseg_blocks 64-wide k-blocks each, zero-filled at each segment's end)
+  const int kblocks = p.conv_rows > 1 ? p.conv_rows * p.kseg_blocks / p.ksub : (p.K + kstep - 1) / kstep;
   // 3xTF32: the tensor core truncates the fp32 accumulator once per instruction, a bias that grows
   // with the number of instructions in a chain (about 7e-9 K relative).  So a tile's K range is cut
   // into chunks of p.chunk_blocks k-blocks; each chunk is accumulated in tensor memory on its own and
@@ -451,34 +452,63 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (long long t = unit0; t < p.num_tiles && ok; t += unit_step) {
-        const TileCoord c = tile_coord(t, p, rank);
-        for (int kb = 0; kb < kblocks; ++kb, ++it) {
-          const int s = it % p.stages;
-          const uint32_t ph = (it / p.stages) & 1u;
-          if (!(ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status))) break;
-          const uint32_t xs = base + (uint32_t)(s * L.stage_bytes);
-          if constexpr (PAIR) {
-            if (rank == 0) mbar_arrive_expect_tx(full_bar(s), 2u * (uint32_t)L.stage_bytes);
-          } else {
-            mbar_arrive_expect_tx(full_bar(s), (uint32_t)L.stage_bytes);
-          }
-          // The sub-blocks of a stage are adjacent in K: consecutive requests for the same matrix
-          // rows ask the DRAM for neighbouring 128-byte lines (out-of-range sub-blocks read as zero).
-          for (int j = 0; j < p.ksub; ++j) {
-            const int k0 = kb * kstep + j * (TF32 ? p.k_plane : kUmmaBlockK);
-            const uint32_t dst = xs + (uint32_t)(j * L.sub_bytes) + L.x_bytes;
-            if constexpr (PAIR) tma_load_3d_pair(dst, &tmap_w, k0, c.n0 + rank * w_rows, p.w_shared ? 0 : c.bt, full_bar(s));
-            else tma_load_3d(dst, &tmap_w, k0, c.n0, p.w_shared ? 0 : c.bt, full_bar(s));
-          }
-          for (int j = 0; j < p.ksub; ++j) {
-            const int k0 = kb * kstep + j * (TF32 ? p.k_plane : kUmmaBlockK);
-            const uint32_t dst = xs + (uint32_t)(j * L.sub_bytes);
-            if constexpr (PAIR) tma_load_3d_pair(dst, &tmap_x, k0, c.m0, c.bt, full_bar(s));
-            else tma_load_3d(dst, &tmap_x, k0, c.m0, c.bt, full_bar(s));
+      // The time from a stage's "empty" signal to its loads going out adds to every refill of the ring, so
+      // whatever can be worked out before the wait is: addresses, coordinates, the byte count.  (Measured: a
+      // dozen more integer instructions after the wait cost c2 and c5 4 %.)  The 2-D convolution's coordinates
+      // get a loop of their own (CONV2D), so that plain GEMMs and 1-D convolutions do not pay for them.
+      auto produce = [&](auto conv2d_tag) {
+        constexpr bool CONV2D = decltype(conv2d_tag)::value;
+        const uint32_t tx = (PAIR ? 2u : 1u) * (uint32_t)L.stage_bytes;
+        const int wrow0 = PAIR ? rank * w_rows : 0;
+        uint32_t s = 0, ph = 0;              // ring slot and its phase, kept incrementally
+        for (long long t = unit0; t < p.num_tiles && ok; t += unit_step) {
+          const TileCoord c = tile_coord(t, p, rank);
+          const int wbt = p.w_shared ? 0 : c.bt;
+          for (int kb = 0; kb < kblocks; ++kb, ++it) {
+            const uint32_t xs = base + s * (uint32_t)L.stage_bytes;
+            const uint32_t fb = full_bar((int)s);
+            int kx[4], xy[4], wy[4], wz[4];  // per sub-block: K coordinate, X row, W's second and third coordinate
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              if constexpr (CONV2D) {
+                // k-block g of the tile lies in filter row g / kseg_blocks: its X rows are the output rows shifted
+                // down by that many image rows, its W rows come from that plane of the filters [S C, R, N]
+                const int g = kb * p.ksub + j, fr = g / p.kseg_blocks;
+                kx[j] = (g - fr * p.kseg_blocks) * kUmmaBlockK;
+                xy[j] = c.m0 + fr * p.conv_width;
+                wy[j] = fr;
+                wz[j] = c.n0 + wrow0;
+              } else {
+                kx[j] = kb * kstep + j * (TF32 ? p.k_plane : kUmmaBlockK);
+                xy[j] = c.m0;
+                wy[j] = c.n0 + wrow0;
+                wz[j] = wbt;
+              }
+            }
+            if (!(ok = mbar_wait(empty_bar((int)s), ph ^ 1u, abort_flag, p.status))) break;
+            if (!PAIR || rank == 0) mbar_arrive_expect_tx(fb, tx);
+            // The sub-blocks of a stage are adjacent in K: consecutive requests for the same matrix
+            // rows ask the DRAM for neighbouring 128-byte lines (out-of-range sub-blocks read as zero).
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              if (j < p.ksub) {
+                const uint32_t dst = xs + (uint32_t)(j * L.sub_bytes) + L.x_bytes;
+                if constexpr (PAIR) tma_load_3d_pair(dst, &tmap_w, kx[j], wy[j], wz[j], fb);
+                else tma_load_3d(dst, &tmap_w, kx[j], wy[j], wz[j], fb);
+              }
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              if (j < p.ksub) {
+                const uint32_t dst = xs + (uint32_t)(j * L.sub_bytes);
+                if constexpr (PAIR) tma_load_3d_pair(dst, &tmap_x, kx[j], xy[j], c.bt, fb);
+                else tma_load_3d(dst, &tmap_x, kx[j], xy[j], c.bt, fb);
+              }
+            if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; }
           }
         }
-      }
+      };
+      if (!TF32 && p.conv_rows > 1) produce(std::true_type{});
+      else produce(std::false_type{});
       if (!ok && !PAIR) {
         // Aborting: let the copies already issued land before the CTA gives its shared memory back.
         // (A pair ends with a cluster-wide barrier and its copies are counted in the leader, so
@@ -497,6 +527,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
     if (lane == 0 && rank == 0) {
       const uint32_t idesc = make_idesc(PAIR ? 2 * kUmmaTileM : kUmmaTileM, p.tile_n, TF32);
       uint32_t it = 0, tcount = 0;       // tcount counts accumulator hand-overs: tiles, or K chunks of tiles (3xTF32)
+      uint32_t slot = 0, sph = 0;        // ring slot and its phase, kept incrementally
       bool ok = true;
       for (long long t = unit0; t < p.num_tiles && ok; t += unit_step)
        for (int kb0 = 0; kb0 < kblocks && ok; kb0 += chunk_blocks, ++tcount) {
@@ -506,14 +537,20 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
         const uint32_t d = tmem_base + buf * 256u;
         const int kb1 = kb0 + chunk_blocks < kblocks ? kb0 + chunk_blocks : kblocks;
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
-          const int s = it % p.stages;
-          const uint32_t ph = (it / p.stages) & 1u;
-          if (!(ok = mbar_wait(full_bar(s), ph, abort_flag, p.status))) break;
+          const int s = (int)slot;
+          // descriptors of the stage's tiles before the wait: the MMAs go out the moment the operands are there
+          const uint32_t xs = base + slot * (uint32_t)L.stage_bytes;
+          uint64_t adesc[4], bdesc[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            adesc[j] = make_smem_desc(xs + (uint32_t)(j * L.sub_bytes));
+            bdesc[j] = make_smem_desc(xs + (uint32_t)(j * L.sub_bytes) + L.x_bytes);
+          }
+          if (!(ok = mbar_wait(full_bar(s), sph, abort_flag, p.status))) break;
           tcgen05_fence_after();
-          const uint32_t xs = base + (uint32_t)(s * L.stage_bytes);
+          if (++slot == (uint32_t)p.stages) { slot = 0; sph ^= 1u; }
           if constexpr (TF32) {
-            const uint64_t a_hi = make_smem_desc(xs), b_hi = make_smem_desc(xs + L.x_bytes);
-            const uint64_t a_lo = make_smem_desc(xs + (uint32_t)L.sub_bytes), b_lo = make_smem_desc(xs + (uint32_t)L.sub_bytes + L.x_bytes);
+            const uint64_t a_hi = adesc[0], b_hi = bdesc[0], a_lo = adesc[1], b_lo = bdesc[1];
 #pragma unroll
             for (int pr = 0; pr < 3; ++pr) {               // the two small products first, then hi * hi
               const uint64_t a0 = pr == 0 ? a_lo : a_hi, b0 = pr == 1 ? b_lo : b_hi;
@@ -524,16 +561,17 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
                 else tcgen05_mma_tf32(d, a0 + 2u * k, b0 + 2u * k, idesc, acc);
               }
             }
-          }
-          for (int j = 0; !TF32 && j < p.ksub; ++j) {
-            const uint64_t a0 = make_smem_desc(xs + (uint32_t)(j * L.sub_bytes));
-            const uint64_t b0 = make_smem_desc(xs + (uint32_t)(j * L.sub_bytes) + L.x_bytes);
+          } else {
 #pragma unroll
-            for (int k = 0; k < kUmmaBlockK / 16; ++k) {   // 16 bf16 = 32 bytes = 2 descriptor address units
-              const uint32_t acc = (kb | j | k) != 0 ? 1u : 0u;
-              if constexpr (PAIR) tcgen05_mma_bf16_pair(d, a0 + 2u * k, b0 + 2u * k, idesc, acc);
-              else tcgen05_mma_bf16(d, a0 + 2u * k, b0 + 2u * k, idesc, acc);
-            }
+            for (int j = 0; j < 4; ++j)
+              if (j < p.ksub) {
+#pragma unroll
+                for (int k = 0; k < kUmmaBlockK / 16; ++k) {   // 16 bf16 = 32 bytes = 2 descriptor address units
+                  const uint32_t acc = (kb | j | k) != 0 ? 1u : 0u;
+                  if constexpr (PAIR) tcgen05_mma_bf16_pair(d, adesc[j] + 2u * k, bdesc[j] + 2u * k, idesc, acc);
+                  else tcgen05_mma_bf16(d, adesc[j] + 2u * k, bdesc[j] + 2u * k, idesc, acc);
+                }
+              }
           }
           if constexpr (PAIR) tcgen05_commit_pair(empty_bar(s)); else tcgen05_commit(empty_bar(s));
         }

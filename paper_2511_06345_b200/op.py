@@ -15,17 +15,19 @@ class FusedGemmReduce:
     X [batch, M, K] and W [batch, N, K] are packed CUDA tensors (bf16 or fp32 as configured).
     With ``conv_taps = R > 1`` (1-D convolution as an implicit GEMM) X is the channels-last input
     [batch, M + R - 1, K / R] (stride s: ``ldx = s * K / R``, signal length (M - 1) s + R) and W the filters [batch, N, K]; ``w_shared=1``: W is one [N, K] matrix
-    for all batch elements.
+    for all batch elements.  ``conv_rows = R > 1``: 2-D convolution, X the channels-last image
+    [batch, H, conv_width, K / (R * conv_taps)], output rows at the image's row pitch (see ``include/fgr.h``).
     """
 
     def __init__(self, batch, M, N, K, dtype, act, scale_kind, reduce, *, scale=1.0, write_y=0, bias_per_batch=0,
-                 device=0, force_path=B.FGR_PATH_AUTO, force_tile_n=0, force_cta_pair=0, force_ksub=0, conv_taps=0, w_shared=0, ldx=0):
+                 device=0, force_path=B.FGR_PATH_AUTO, force_tile_n=0, force_cta_pair=0, force_ksub=0, conv_taps=0, w_shared=0, ldx=0, conv_rows=0,
+                 conv_width=0):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required: this operator has no CPU path")
         self.desc = B.make_desc(batch, M, N, K, dtype, act, scale_kind, reduce, scale=scale, write_y=write_y,
                                 bias_per_batch=bias_per_batch, device=device, force_path=force_path,
                                 force_tile_n=force_tile_n, force_cta_pair=force_cta_pair, force_ksub=force_ksub,
-                                conv_taps=conv_taps, w_shared=w_shared, ldx=ldx)
+                                conv_taps=conv_taps, w_shared=w_shared, ldx=ldx, conv_rows=conv_rows, conv_width=conv_width)
         self.handle = B.fgr_create(self.desc)
         self.plan = B.fgr_get_plan(self.handle)
         self.device = torch.device("cuda", device)

@@ -44,7 +44,7 @@ def run_gpu(p: gi.Problem, force_path=0, force_tile_n=0, device=0, tensors=None,
     op = fgr.FusedGemmReduce(p.batch, p.M, p.N, p.K, p.dtype, p.act, p.scale_kind, p.reduce, scale=p.scale,
                              write_y=p.write_y, bias_per_batch=p.bias_per_batch, device=device,
                              force_path=force_path, force_tile_n=force_tile_n, force_cta_pair=force_cta_pair, force_ksub=force_ksub,
-                             conv_taps=p.conv_taps, w_shared=p.w_shared,
+                             conv_taps=p.conv_taps, w_shared=p.w_shared, conv_rows=p.conv_rows, conv_width=p.conv_width,
                              ldx=(p.conv_stride * (p.K // p.conv_taps) if p.conv_taps > 1 and p.conv_stride > 1 else 0))
     X, W, b, s = tensors if tensors is not None else to_device(p, "cuda:%d" % device)
     R = None

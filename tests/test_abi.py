@@ -34,7 +34,7 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_struct_layout_matches_header():
-    assert ctypes.sizeof(fgr.fgr_desc) == 128      # the value sizeof(fgr_desc) has in C (gcc, x86-64)
+    assert ctypes.sizeof(fgr.fgr_desc) == 136      # the value sizeof(fgr_desc) has in C (gcc, x86-64)
     assert ctypes.sizeof(fgr.fgr_plan_info) == 72
     assert fgr.fgr_status_string(0) == "ok" and "wait" in fgr.fgr_status_string(fgr.FGR_ERR_DEVICE_TIMEOUT)
     assert fgr.fgr_path_name(fgr.FGR_PATH_UMMA_STREAM_W) == "umma_stream_w"
