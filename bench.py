@@ -684,7 +684,7 @@ def run_nshard(args, ctx):
 # DRAM bytes per launch of the main kernel from ncu (dram__bytes_read.sum + dram__bytes_write.sum), one
 # capture per workload of the kernel as it stands; a workload without a capture of the current kernel
 # reports null.
-TRAFFIC = {"c2": 88.32e6, "c3": 184.46e6, "c4": 274.77e6, "c5": 70.93e6, "g2": 271.83e6,
+TRAFFIC = {"c2": 90.43e6, "c3": 183.49e6, "c4": 274.99e6, "c5": 70.69e6, "g2": 271.83e6,
            "r_max": 138.23e6, "r_lse": 139.97e6, "r_softmax": 224.41e6, "r_meanvar": 138.14e6,
            "r_max_long": 138.70e6, "r_lse_long": 140.99e6, "f2": 769.50e6, "v2": 124.35e6}
 
