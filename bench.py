@@ -39,7 +39,10 @@ HBM_BOUND = {"c4", "g2"}
 EXTRA_CONFIGS = {"g2": ("c4", dict(M=2)),     # c4's shapes and epilogue with M = 2
                  "f2": ("c2", dict(dtype=0)),  # c2's shapes and epilogue with fp32 inputs and outputs: the 3xTF32 path
                  # 1-D convolution with c2's epilogue: 8 signals of 2051 x 512 channels, 4096 filters of 4 taps (shared)
-                 "v2": ("c2", dict(batch=8, M=2048, N=4096, K=2048, conv_taps=4, w_shared=1))}
+                 "v2": ("c2", dict(batch=8, M=2048, N=4096, K=2048, conv_taps=4, w_shared=1)),
+                 # 2-D convolution with c2's epilogue: 16 images of 66 x 66 x 64 channels, 1024 shared filters of 3 x 3
+                 # (64 x 64 outputs per image at the image's row pitch: M = 63 * 66 + 64 rows, 3 % of them unused)
+                 "v3": ("c2", dict(batch=16, M=63 * 66 + 64, N=1024, K=3 * 3 * 64, conv_rows=3, conv_taps=3, conv_width=66, w_shared=1))}
 
 
 def make_cfg(name, **kw):
@@ -227,7 +230,8 @@ def shape_keys(cfg, p):
     import fgr_inputs as gi
     return {"workload": cfg, "batch": p.batch, "M": p.M, "N": p.N, "K": p.K, "act": ACT_NAMES[p.act],
             "scale": SCALE_NAMES[p.scale_kind], "reduce": REDUCE_NAMES[p.reduce],
-            "write_y": int(bool(p.write_y) or p.reduce == gi.RED_SOFTMAX), "conv_taps": p.conv_taps, "w_shared": p.w_shared}
+            "write_y": int(bool(p.write_y) or p.reduce == gi.RED_SOFTMAX), "conv_taps": p.conv_taps, "w_shared": p.w_shared,
+            "conv_rows": p.conv_rows, "conv_width": p.conv_width}
 
 
 def run_reference(args):
@@ -327,7 +331,7 @@ def measure_fused(cfg, args, ctx, with_e2e=True, with_cpu=True):
 
     desc = fgr.make_desc(p.batch, p.M, p.N, p.K, p.dtype, p.act, p.scale_kind, p.reduce, scale=p.scale,
                          write_y=p.write_y, bias_per_batch=p.bias_per_batch, device=local_rank,
-                         conv_taps=p.conv_taps, w_shared=p.w_shared)
+                         conv_taps=p.conv_taps, w_shared=p.w_shared, conv_rows=p.conv_rows, conv_width=p.conv_width)
     h = fgr.fgr_create(desc)
     plan = fgr.fgr_get_plan(h)
     ws_bytes = fgr.fgr_workspace_bytes(h)

@@ -113,6 +113,8 @@ def test_bench_extra_workloads_are_well_formed():
     v2 = bench.make_cfg("v2", materialize=False)
     assert (v2.batch, v2.M, v2.N, v2.K, v2.conv_taps, v2.w_shared) == (8, 2048, 4096, 2048, 4, 1)
     assert v2.flop == 2.0 * 8 * 2048 * 4096 * 2048
+    v3 = bench.make_cfg("v3", materialize=False)
+    assert (v3.batch, v3.M, v3.N, v3.K, v3.conv_rows, v3.conv_taps, v3.conv_width) == (16, 63 * 66 + 64, 1024, 576, 3, 3, 66)
     g2 = bench.make_cfg("g2", materialize=False)
     assert (g2.M, g2.N, g2.K) == (2, 16384, 8192)
     for name in ("c2", "c3", "c4", "c5", "f2", "v2", "g2"):
