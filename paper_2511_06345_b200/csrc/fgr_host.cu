@@ -301,9 +301,8 @@ int make_plan(const fgr_desc& d, int num_sms, fgr_plan_info* info, Params* pp) {
     int ksub = tf32 ? 2 : d.force_ksub;   // 3xTF32: the two sub-blocks of a stage are the hi and lo planes
     if (!ksub) ksub = (d.K > kUmmaBlockK && umma_smem_layout(w_rows, 3, 2).total <= kSmemLimit) ? 2 : 1;
     while (!tf32 && ksub > 1 && umma_smem_layout(w_rows, 2, ksub).total > kSmemLimit) --ksub;
-    if (conv2d) {   // a ring stage must not straddle two filter rows unevenly: whole k-blocks, ksub of them per stage
-      while (ksub > 1 && (d.conv_rows * p.kseg_blocks) % ksub != 0) --ksub;
-    }
+    // (2-D convolution: a stage is ksub whole k-blocks of the R * kseg_blocks the tile has; when that number is not a
+    //  multiple of ksub the last stage's surplus sub-blocks lie beyond the last filter row and read as zero)
     p.ksub = ksub;
     p.k_plane = tf32 ? (d.K + 31) / 32 * 32 : 0;
     p.chunk_blocks = kTf32ChunkBlocks;

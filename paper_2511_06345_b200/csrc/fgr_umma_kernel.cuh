@@ -407,7 +407,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kstep = TF32 ? kUmmaBlockK / 2 : kUmmaBlockK * p.ksub;   // K elements per ring stage (128-byte rows)
   // (2-D convolution: conv_rows segments of kseg_blocks 64-wide k-blocks each, zero-filled at each segment's end)
-  const int kblocks = p.conv_rows > 1 ? p.conv_rows * p.kseg_blocks / p.ksub : (p.K + kstep - 1) / kstep;
+  const int kblocks = p.conv_rows > 1 ? (p.conv_rows * p.kseg_blocks + p.ksub - 1) / p.ksub : (p.K + kstep - 1) / kstep;
   // 3xTF32: the tensor core truncates the fp32 accumulator once per instruction, a bias that grows
   // with the number of instructions in a chain (about 7e-9 K relative).  So a tile's K range is cut
   // into chunks of p.chunk_blocks k-blocks; each chunk is accumulated in tensor memory on its own and
