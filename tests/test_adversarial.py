@@ -156,6 +156,37 @@ def test_host_buffer_entry_point_in_chunks(cuda_device):
         fgr.fgr_destroy(h)
 
 
+def test_softmax_back_to_back_runs_share_a_workspace(cuda_device):
+    """The softmax normalise kernel runs beside the main kernel and follows per-row-block completion counters in
+    the workspace, which the last normalise CTA zeroes.  Sixty runs in a row on one stream and one workspace,
+    alternating two problems (so the next run's main kernel is resident while this run's normalise kernel is
+    still working): every run must reproduce, bit for bit, what the same problem gives when run alone, and
+    that must match the oracle."""
+    probs = [gi.make_config("c3", M=1100, N=2056, K=264, scale=2.0, seed=s) for s in (81, 82)]
+    desc = fgr.make_desc(1, 1100, 2056, 264, probs[0].dtype, probs[0].act, probs[0].scale_kind, probs[0].reduce, scale=2.0)
+    h = fgr.fgr_create(desc)
+    assert fgr.fgr_get_plan(h).path == fgr.FGR_PATH_UMMA_TILED
+    ws = torch.empty(fgr.fgr_workspace_bytes(h), dtype=torch.uint8, device="cuda")
+    dev = [to_device(p) for p in probs]
+    stream = torch.cuda.current_stream().cuda_stream
+    alone = []
+    for (X, W, b, s_) in dev:
+        P = torch.empty((1100, 2056), dtype=torch.bfloat16, device="cuda")
+        fgr.fgr_run(h, X, W, b, s_, P, None, ws, ws.numel(), stream)
+        assert fgr.fgr_get_status(h) == fgr.FGR_OK
+        alone.append(P.clone())
+    outs = [torch.empty((1100, 2056), dtype=torch.bfloat16, device="cuda") for _ in range(60)]
+    for i, P in enumerate(outs):
+        X, W, b, s_ = dev[i % 2]
+        fgr.fgr_run(h, X, W, b, s_, P, None, ws, ws.numel(), stream)
+    assert fgr.fgr_get_status(h) == fgr.FGR_OK
+    for i, P in enumerate(outs):
+        assert torch.equal(P.view(torch.int16), alone[i % 2].view(torch.int16)), "run %d differs" % i
+    for p, P in zip(probs, alone):
+        compare(p, P.float().cpu().numpy().astype(np.float64), None)
+    fgr.fgr_destroy(h)
+
+
 def test_null_and_misaligned_pointers_are_rejected(cuda_device):
     p = gi.make_config("c2", M=130, N=264, K=72)
     X, W, b, s = to_device(p)
